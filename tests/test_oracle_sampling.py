@@ -398,3 +398,50 @@ def test_verify_window_first_rejection_and_alpha_mixture():
         n_rows += L - a
     # alpha = 1 is the coupling itself; more coupling -> more identical redraws (Sec. 5.1)
     assert n_same[1.0] > n_same[0.5] > n_same[0.0]
+
+
+@pytest.mark.parametrize("alpha", [0.0, 0.3, 0.75, 1.0])
+def test_alpha_coin_rate_and_coupling_cost(alpha):
+    """Algorithm 5 (alpha-coupling): every row beyond the committed prefix keeps its coupled
+    redraft with probability alpha and takes an independent draw from p otherwise, so that
+    Pr[X = Y] = alpha (1 - TV(p, q)) + (1 - alpha) sum_x p(x) q(x)   (Sec. 5.1, coupling strength).
+    The rate of the coin itself is counted on rows where the two candidate outputs differ (what the
+    row received then says which branch ran); the cost is counted on all rows. Both within five
+    standard deviations over more than 10^5 (position, iteration) keys: a coin firing with alpha/2,
+    alpha^2 or 1 - alpha fails for every alpha strictly inside (0, 1), and at the ends."""
+    L, V, seed = 33, 8, 77
+    p = np.array([9, 1, 14, 3, 0, 6, 11, 4], dtype=np.uint32)
+    q = np.array([2, 12, 5, 3, 7, 0, 9, 10], dtype=np.uint32)
+    Zp, Zq = int(p.sum()), int(q.sum())
+    P, Q = p / Zp, q / Zq
+    # row 0 always rejects (its draft has no mass under p0): a = 1, so rows 1..L-1 all meet the coin
+    p0 = np.array([1, 1, 1, 1, 0, 0, 0, 0], dtype=np.uint32)
+    q0 = np.array([0, 0, 0, 0, 1, 1, 1, 1], dtype=np.uint32)
+    Wp = np.vstack([p0] + [p] * (L - 1))
+    Wq = np.vstack([q0] + [q] * (L - 1))
+    Zps = np.array([4] + [Zp] * (L - 1), dtype=np.uint64)
+    Zqs = np.array([4] + [Zq] * (L - 1), dtype=np.uint64)
+    rng = np.random.default_rng(int(alpha * 100) + 1)
+    n_dist = n_kept = n_rows = n_same = 0
+    for trial in range(3200):
+        pos0, it = 1000 + 40 * trial, trial % 97
+        X = np.array([5] + [oracle.sample(q, Zq, int(u)) for u in rng.integers(0, N24, L - 1)], dtype=np.int32)
+        a_mc, _, Y_mc = oracle.verify_window(Wp, Zps, Wq, Zqs, X, pos0, it, seed, mode=0)
+        a, _, Y = oracle.verify_window(Wp, Zps, Wq, Zqs, X, pos0, it, seed, mode=2, alpha=alpha)
+        assert a_mc == 1 and a == 1 and Y[0] == Y_mc[0]
+        for k in range(1, L):
+            Ui = oracle.noise_u24(seed, oracle.NOISE_INDEP, 0, pos0 + k, it)
+            y_ind = oracle.sample(p, Zp, Ui)
+            assert Y[k] in (Y_mc[k], y_ind)
+            if Y_mc[k] != y_ind:
+                n_dist += 1
+                n_kept += int(Y[k] == Y_mc[k])
+        n_rows += L - 1
+        n_same += int((Y[1:] == X[1:]).sum())
+    assert n_rows >= 100_000 and n_dist >= 50_000
+    assert abs(n_kept - alpha * n_dist) <= 5 * math.sqrt(alpha * (1 - alpha) * n_dist)
+    if alpha in (0.0, 1.0):
+        assert n_kept == int(alpha) * n_dist
+    tvd = 0.5 * np.abs(P - Q).sum()
+    cost = alpha * (1.0 - tvd) + (1.0 - alpha) * float((P * Q).sum())
+    assert abs(n_same / n_rows - cost) <= 5 * math.sqrt(cost * (1 - cost) / n_rows)
