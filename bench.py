@@ -251,8 +251,6 @@ def run_scd(args, shape):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     scd.lib()                                            # fails loudly if libscd.so is missing
-    if args.gemm_splits or args.gemm_stages:
-        scd.scd_gemm_tune(args.gemm_splits, args.gemm_stages)
 
     B = args.batch
     S = 2 if shape["cfg_lambda"] != 0.0 else 1
@@ -261,6 +259,8 @@ def run_scd(args, shape):
     max_seq = P + N + L
     w = synth.make_weights(shape, seed=1234, device="cuda")
     model = scd.Model(shape, w, max_seq=max_seq)
+    if args.gemm_splits or args.gemm_stages:
+        model.scd_model_gemm_tune(args.gemm_splits, args.gemm_stages)
     cond, uncond = synth.make_prompt(shape, batch=B)
     prompts = np.concatenate([cond, uncond]) if S == 2 else cond
 

@@ -42,7 +42,8 @@ enum {
     SCD_ERR_CAPACITY = -3,    /* would exceed max_seq / window / scratch capacity */
     SCD_ERR_STATE = -4,       /* call out of order (e.g. step before prefill) */
     SCD_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed; see scd_last_error() */
-    SCD_ERR_TIMEOUT = -6,     /* a bounded device-side wait gave up */
+    SCD_ERR_TIMEOUT = -6,     /* a bounded device-side wait gave up; the session's error word stays set
+                                 until the next scd_prefill, which clears it: re-prefill or recreate */
     SCD_ERR_UNSUPPORTED = -7  /* valid request that the library does not implement */
 };
 
@@ -120,7 +121,9 @@ const char *scd_strerror(int code);
 const char *scd_last_error(void);
 
 /* ---- model ------------------------------------------------------------------------------
- * scd_init_model: validates the shape, records the borrowed weight pointers, builds the RoPE
+ * scd_init_model: the model p_theta that Algorithm 6 REQUIREs (a Llama-style decoder; the paper treats it
+ * as a black box that yields p_theta(. | X_{0:j-1}) for all window positions in one pass, Sec. 2.2).
+ * Validates the shape, records the borrowed weight pointers, builds the RoPE
  * table and the TMA descriptors of the weight matrices on the current CUDA device.
  * Errors: SCD_ERR_ARG (null), SCD_ERR_SHAPE (odd head_dim, heads not divisible, sizes <= 0;
  * bf16 models additionally need d_model, d_ffn and n_heads*head_dim to be multiples of 64),
@@ -129,6 +132,8 @@ int scd_init_model(const scd_model_config_t *cfg, const scd_weights_t *weights, 
 int scd_free_model(scd_model_t *model);
 
 /* ---- session ----------------------------------------------------------------------------
+ * scd_session_create: the state Algorithm 6 keeps between iterations (REQUIRE: draft length L, maximum
+ * sequence length; its loop variables i, t, the drafts X and the draft distributions p^(t)).
  * A session holds the KV cache (paged), the window state (drafts, draft distributions, position
  * and iteration counters - all resident on the device) and scratch activations for one decode
  * batch. Allocates device memory (cudaMalloc); free with scd_session_free. */
@@ -149,46 +154,15 @@ int scd_prefill(scd_session_t *session, const int32_t *prompt_ids, int32_t P, in
  * Fully asynchronous; all state stays on the device. */
 int scd_step(scd_session_t *session, void *stream);
 
-/* scd_step_profile: one iteration exactly like scd_step, with a CUDA event recorded on `stream`
- * in front of every kernel; the device time between consecutive events is ADDED to
- * ms_by_class[c] and the kernel count to launches_by_class[c] ([host] arrays of
- * SCD_PROF_CLASSES entries, which the caller zeroes), c being the class of the kernel launched
- * between them. Blocking. Used to attribute the time of an iteration (Sec. 4.3, latency
- * breakdown per NFE step) to its kernels. */
-enum { SCD_PROF_EMBED = 0, SCD_PROF_RMSNORM, SCD_PROF_GEMM_QKV, SCD_PROF_ROPE_KV, SCD_PROF_ATTENTION,
-       SCD_PROF_GEMM_O, SCD_PROF_GEMM_GATE_UP, SCD_PROF_GEMM_DOWN, SCD_PROF_GEMM_LM_HEAD,
-       SCD_PROF_VERIFY, SCD_PROF_OTHER, SCD_PROF_CLASSES };
-int scd_step_profile(scd_session_t *session, float *ms_by_class, int32_t *launches_by_class,
-                     void *stream);
-
-/* scd_kernel_launches: number of CUDA kernels this process has enqueued through the library. */
-int64_t scd_kernel_launches(void);
-/* scd_autotune: measures, for this model and this session's window shape, how many K slices
- * (1..8, = cluster size) make each kind of weight GEMM of the layer - QKV, output projection,
- * gate/up, down - fastest inside a whole window forward, and keeps the winners for every later
- * launch on this model (all its sessions). It runs a few dozen window forwards without verify and
- * without commit: tokens, counters and the committed KV cache do not change. k_splits_out (host,
- * 4 entries, optional) receives the choices (0: the built-in rule stays). The slicing changes the
- * order of the fp32 additions of a GEMM, so logits may differ in their last bits from an untuned
- * run, and with them the sampled tokens: call it (or not) consistently where runs must be
- * comparable token by token. fp32 models: no-op. Blocking. Errors: SCD_ERR_STATE before
- * scd_prefill, SCD_ERR_CUDA. */
-int scd_autotune(scd_session_t *session, int32_t *k_splits_out, void *stream);
-/* Like scd_step_profile (one iteration, same arrays, same classes, blocking), but without events
- * between the kernels: the GEMM and attention kernels write the GPU timer at CTA entry and exit
- * into a device buffer, so neighbouring kernels overlap exactly as in scd_step. The time from the
- * end of the previous stamped kernel to the end of a kernel is charged to that kernel's class; the
- * embedding gather and the verify kernel leave no stamps and are not counted (their classes stay 0).
- * The first call allocates the stamp buffer (a few MiB, freed with the session). */
-int scd_step_timeline(scd_session_t *session, float *ms_by_class, int32_t *launches_by_class, void *stream);
-
-/* scd_step_result: waits for the stream, then copies out per-sequence counters.
+/* scd_step_result: the loop variables of Algorithm 6 after an iteration (i <- Accept + 1): waits for
+ * the stream, then copies out per-sequence counters.
  * n_committed[b] = tokens committed by the LAST step, n_known[b] = prompt + committed tokens,
  * kv_len[b] = committed KV entries (always n_known - 1). Any pointer may be NULL. [host][B] */
 int scd_step_result(scd_session_t *session, int32_t *n_committed, int32_t *n_known,
                     int32_t *kv_len, void *stream);
 
-/* scd_generate: runs iterations until every sequence holds n_total tokens (set by prefill),
+/* scd_generate: the While loop of Algorithm 6 ("while i < N"; Algorithm 7 in SCD_MODE_SCD_GS, Algorithm 2
+ * in SCD_MODE_SJD): runs iterations until every sequence holds n_total tokens (set by prefill),
  * then copies the generated tokens to out_tokens [host] int32 [B, n_new] and fills stats
  * [host] (may be NULL). Blocking. */
 int scd_generate(scd_session_t *session, int32_t *out_tokens, scd_stats_t *stats, void *stream);
@@ -205,7 +179,9 @@ int scd_read_tokens(scd_session_t *session, int32_t first, int32_t count, int32_
  *   q_logits      [dev] f32 [B, L, V]     draft logits, post-processed with the same temperature
  *                                         and top-k (no guidance); NULL = every row is fresh
  *                                         (uniform over the allowed ids)
- *   draft_ids     [dev] i32 [B, L]        X_j, assumed drawn from q_j
+ *   draft_ids     [dev] i32 [B, L]        X_j, drawn from q_j: inside the allowed range with q_j(X_j) > 0.
+ *                                         (A draft without mass under p_j is rejected whatever q_j says,
+ *                                         so no id outside the support of p is ever committed.)
  *   positions     [dev] i64 [B]           global position of window row 0 of each sequence
  *   iteration                              t (noise key)
  *   n_commit      [dev] i32 [B]           out: a = tokens committed (1..L)
@@ -232,14 +208,18 @@ int scd_verify(const scd_decode_config_t *cfg, int32_t V, const float *p_logits,
  * library: a file-scope device array of scd_verify_noalloc_max_bytes() bytes (16 MiB) that
  * every GPU context loading the library holds until the process exits.
  *   - Arguments, outputs and results are exactly those of scd_verify, minus `workspace`.
- *   - Neither this call nor anything it calls allocates or frees memory (no cudaMalloc / cudaFree,
- *     no allocating library routine). The caller still supplies all inputs and outputs.
+ *   - The call issues no cudaMalloc / cudaFree and no allocating library routine; the caller still
+ *     supplies all inputs and outputs.
  *   - A request whose scratch (scd_verify_workspace_bytes) exceeds the built-in buffer returns
  *     SCD_ERR_CAPACITY and launches nothing; e.g. B = 1 or 2 with L = 32, V = 16384 fit,
  *     B = 8 does not: use scd_verify with your own workspace there.
- *   - The first call on each device looks up the buffer's device address (one
- *     cudaGetSymbolAddress with that device current). Make that first call outside any stream
- *     capture.
+ *   - The FIRST call on each device is a warm-up and belongs to start-up: it looks up the buffer's
+ *     device address (one cudaGetSymbolAddress with that device current), and with CUDA's lazy module
+ *     loading it is also the moment the runtime loads the kernels on that device and gives the 16 MiB
+ *     array its memory - so that first call may synchronise, take memory, or fail where memory is
+ *     already short. Make it (any small problem will do) before device memory is handed to your own
+ *     pool and outside any stream capture; from the second call on nothing is allocated. The address
+ *     is cached per device ordinal for the life of the process (cudaDeviceReset invalidates it).
  *   - All calls on a device share the one buffer, which keeps whatever the previous call left
  *     in it; the part that must start at zero is cleared on `stream` before the kernel. Two
  *     calls that can overlap on the GPU (different streams, no ordering between them) race on
@@ -260,30 +240,6 @@ int scd_verify_noalloc(const scd_decode_config_t *cfg, int32_t V, const float *p
  * is recomputed by the next forward). Positions beyond max_seq are neither written nor read. */
 int scd_forward_window(scd_session_t *session, const int32_t *ids, int32_t M, float *logits,
                        float *hidden, int32_t commit, void *stream);
-
-/* scd_debug_read: copies a piece of session state to host memory, for step-level parity tests.
- * what = 0: the logits of the last step, f32 [S*B, L, V]; what = 1: the current drafts,
- * i32 [B, L]. `bytes` must equal the size of that piece. Blocking. */
-int scd_debug_read(scd_session_t *session, int32_t what, void *out, int64_t bytes, void *stream);
-
-/* scd_noise_u24: the counter-based noise of the sampler, for bit-exactness tests.
- * out[i] = top 24 bits of word 0 of Philox4x32-10(key = seed,
- *          counter = (sub, positions[i], iteration, noise_stream | batch << 8)). [dev] arrays. */
-int scd_noise_u24(uint64_t seed, uint32_t noise_stream, uint32_t batch, const int64_t *positions,
-                  uint32_t iteration, uint32_t sub, int64_t n, uint32_t *out, void *stream);
-
-/* scd_gemm_bf16: the tcgen05 weight-streaming GEMM alone, y[M,N] = x[M,K] * w[N,K]^T with fp32
- * accumulation in tensor memory. x, w [dev] bf16 row-major, y [dev] f32. M <= 256;
- * K % 64 == 0; N % 8 == 0. workspace: [dev] scratch of scd_gemm_workspace_bytes(M, N, K)
- * bytes. */
-/* The workspace must be zero-filled before its first use (it holds the split-K tickets and an
- * error word, both left at zero by every call). scd_gemm_tune overrides, for benchmarking, the
- * number of K slices and ring stages every later GEMM launch of this process picks (0 = automatic);
- * set it before creating sessions. */
-int64_t scd_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K);
-int scd_gemm_tune(int32_t k_splits, int32_t stages);
-int scd_gemm_bf16(const void *x, const void *w, float *y, int32_t M, int32_t N, int32_t K,
-                  void *workspace, void *stream);
 
 #ifdef __cplusplus
 }

@@ -247,7 +247,9 @@ int oracle_mrs(const uint32_t *Wp, uint64_t Zp, const uint32_t *Wq, uint64_t Zq,
 {
     u128 lhs = (u128)(U_acc + 1u) * Wq[X] * Zp;
     u128 rhs = ((u128)Wp[X] * Zq) << 24;
-    if (lhs <= rhs) { *Y = X; return 1; }
+    /* p(X) = 0 is never accepted (u > 0); this also covers p(X) = q(X) = 0, which X ~ q excludes and
+     * where the inequality would read 0 <= 0: a sampler of p must not emit an id without mass. */
+    if (Wp[X] != 0 && lhs <= rhs) { *Y = X; return 1; }
     u128 R = 0;
     for (int v = 0; v < V; ++v) {
         u128 a = (u128)Wp[v] * Zq, b = (u128)Wq[v] * Zp;

@@ -22,7 +22,7 @@ EXPORTS = (
     "scd_strerror", "scd_last_error", "scd_init_model", "scd_free_model", "scd_session_create",
     "scd_session_free", "scd_prefill", "scd_step", "scd_step_result", "scd_generate",
     "scd_read_tokens", "scd_verify_workspace_bytes", "scd_verify", "scd_forward_window",
-    "scd_noise_u24", "scd_gemm_workspace_bytes", "scd_gemm_bf16", "scd_debug_read", "scd_gemm_tune",
+    "scd_noise_u24", "scd_gemm_workspace_bytes", "scd_gemm_bf16", "scd_debug_read", "scd_model_gemm_tune", "scd_gemm_bf16_shaped", "scd_selftest_device_once",
     "scd_step_profile", "scd_step_timeline", "scd_autotune", "scd_kernel_launches", "scd_verify_noalloc", "scd_verify_noalloc_max_bytes",
 )
 
@@ -99,44 +99,46 @@ def _declare(l):
     l.scd_noise_u24.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, vp, C.c_uint32, C.c_uint32,
                                 C.c_int64, vp, vp]
     l.scd_noise_u24.restype = C.c_int
-    if hasattr(l, "scd_init_model"):
-        l.scd_init_model.argtypes = [C.POINTER(ModelConfig), C.POINTER(Weights), C.POINTER(C.c_void_p)]
-        l.scd_init_model.restype = C.c_int
-        l.scd_free_model.argtypes = [vp]
-        l.scd_free_model.restype = C.c_int
-        l.scd_session_create.argtypes = [vp, C.POINTER(DecodeConfig), C.POINTER(C.c_void_p)]
-        l.scd_session_create.restype = C.c_int
-        l.scd_session_free.argtypes = [vp]
-        l.scd_session_free.restype = C.c_int
-        l.scd_prefill.argtypes = [vp, vp, C.c_int32, C.c_int32, vp]
-        l.scd_prefill.restype = C.c_int
-        l.scd_step.argtypes = [vp, vp]
-        l.scd_step.restype = C.c_int
-        l.scd_step_result.argtypes = [vp, vp, vp, vp, vp]
-        l.scd_step_result.restype = C.c_int
-        l.scd_generate.argtypes = [vp, vp, C.POINTER(Stats), vp]
-        l.scd_generate.restype = C.c_int
-        l.scd_read_tokens.argtypes = [vp, C.c_int32, C.c_int32, vp, vp]
-        l.scd_read_tokens.restype = C.c_int
-        l.scd_forward_window.argtypes = [vp, vp, C.c_int32, vp, vp, C.c_int32, vp]
-        l.scd_forward_window.restype = C.c_int
-        l.scd_debug_read.argtypes = [vp, C.c_int32, vp, C.c_int64, vp]
-        l.scd_debug_read.restype = C.c_int
-        l.scd_step_profile.argtypes = [vp, vp, vp, vp]
-        l.scd_step_profile.restype = C.c_int
-        l.scd_autotune.argtypes = [vp, vp, vp]
-        l.scd_autotune.restype = C.c_int
-        l.scd_step_timeline.argtypes = [vp, vp, vp, vp]
-        l.scd_step_timeline.restype = C.c_int
-        l.scd_kernel_launches.argtypes = []
-        l.scd_kernel_launches.restype = C.c_int64
-    if hasattr(l, "scd_gemm_bf16"):
-        l.scd_gemm_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
-        l.scd_gemm_workspace_bytes.restype = C.c_int64
-        l.scd_gemm_bf16.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, C.c_int32, vp, vp]
-        l.scd_gemm_bf16.restype = C.c_int
-        l.scd_gemm_tune.argtypes = [C.c_int32, C.c_int32]
-        l.scd_gemm_tune.restype = C.c_int
+    l.scd_init_model.argtypes = [C.POINTER(ModelConfig), C.POINTER(Weights), C.POINTER(C.c_void_p)]
+    l.scd_init_model.restype = C.c_int
+    l.scd_free_model.argtypes = [vp]
+    l.scd_free_model.restype = C.c_int
+    l.scd_session_create.argtypes = [vp, C.POINTER(DecodeConfig), C.POINTER(C.c_void_p)]
+    l.scd_session_create.restype = C.c_int
+    l.scd_session_free.argtypes = [vp]
+    l.scd_session_free.restype = C.c_int
+    l.scd_prefill.argtypes = [vp, vp, C.c_int32, C.c_int32, vp]
+    l.scd_prefill.restype = C.c_int
+    l.scd_step.argtypes = [vp, vp]
+    l.scd_step.restype = C.c_int
+    l.scd_step_result.argtypes = [vp, vp, vp, vp, vp]
+    l.scd_step_result.restype = C.c_int
+    l.scd_generate.argtypes = [vp, vp, C.POINTER(Stats), vp]
+    l.scd_generate.restype = C.c_int
+    l.scd_read_tokens.argtypes = [vp, C.c_int32, C.c_int32, vp, vp]
+    l.scd_read_tokens.restype = C.c_int
+    l.scd_forward_window.argtypes = [vp, vp, C.c_int32, vp, vp, C.c_int32, vp]
+    l.scd_forward_window.restype = C.c_int
+    l.scd_debug_read.argtypes = [vp, C.c_int32, vp, C.c_int64, vp]
+    l.scd_debug_read.restype = C.c_int
+    l.scd_step_profile.argtypes = [vp, vp, vp, vp]
+    l.scd_step_profile.restype = C.c_int
+    l.scd_autotune.argtypes = [vp, vp, vp]
+    l.scd_autotune.restype = C.c_int
+    l.scd_step_timeline.argtypes = [vp, vp, vp, vp]
+    l.scd_step_timeline.restype = C.c_int
+    l.scd_kernel_launches.argtypes = []
+    l.scd_kernel_launches.restype = C.c_int64
+    l.scd_gemm_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
+    l.scd_gemm_workspace_bytes.restype = C.c_int64
+    l.scd_gemm_bf16.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, C.c_int32, vp, vp]
+    l.scd_gemm_bf16.restype = C.c_int
+    l.scd_gemm_bf16_shaped.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, vp, vp]
+    l.scd_gemm_bf16_shaped.restype = C.c_int
+    l.scd_model_gemm_tune.argtypes = [vp, C.c_int32, C.c_int32]
+    l.scd_model_gemm_tune.restype = C.c_int
+    l.scd_selftest_device_once.argtypes = []
+    l.scd_selftest_device_once.restype = C.c_int
 
 
 def _check(rc):
@@ -227,8 +229,9 @@ def scd_gemm_workspace_bytes(M, N, K) -> int:
     return int(n)
 
 
-def scd_gemm_bf16(x, w, y=None, workspace=None, stream=None):
-    """y[M,N] = x[M,K] @ w[N,K]^T (bf16 in, fp32 out) on the tcgen05 weight-streaming kernel."""
+def scd_gemm_bf16(x, w, y=None, workspace=None, stream=None, k_splits=0, stages=0):
+    """y[M,N] = x[M,K] @ w[N,K]^T (bf16 in, fp32 out) on the tcgen05 weight-streaming kernel
+    (scd_gemm_bf16_shaped when a launch shape is given)."""
     M, K = x.shape
     N = w.shape[0]
     assert x.dtype == torch.bfloat16 and w.dtype == torch.bfloat16 and w.shape[1] == K
@@ -238,7 +241,11 @@ def scd_gemm_bf16(x, w, y=None, workspace=None, stream=None):
     if workspace is None:
         workspace = torch.zeros(max(scd_gemm_workspace_bytes(M, N, K), 256), dtype=torch.uint8,
                                 device=x.device)
-    _check(lib().scd_gemm_bf16(_ptr(x), _ptr(w), _ptr(y), M, N, K, _ptr(workspace), _stream(stream)))
+    if k_splits or stages:
+        _check(lib().scd_gemm_bf16_shaped(_ptr(x), _ptr(w), _ptr(y), M, N, K, k_splits, stages, _ptr(workspace),
+                                          _stream(stream)))
+    else:
+        _check(lib().scd_gemm_bf16(_ptr(x), _ptr(w), _ptr(y), M, N, K, _ptr(workspace), _stream(stream)))
     return y
 
 
@@ -246,8 +253,8 @@ def scd_kernel_launches() -> int:
     return int(lib().scd_kernel_launches())
 
 
-def scd_gemm_tune(k_splits: int = 0, stages: int = 0):
-    _check(lib().scd_gemm_tune(k_splits, stages))
+def scd_selftest_device_once() -> int:
+    return int(lib().scd_selftest_device_once())
 
 
 # ------------------------------------------------------------------------------------ model / session
@@ -283,6 +290,9 @@ class Model:
         h = C.c_void_p()
         _check(lib().scd_init_model(C.byref(cfg), C.byref(w), C.byref(h)))
         self.handle = h
+
+    def scd_model_gemm_tune(self, k_splits: int = 0, stages: int = 0):
+        _check(lib().scd_model_gemm_tune(self.handle, k_splits, stages))
 
     def close(self):
         if getattr(self, "handle", None):

@@ -155,13 +155,18 @@ void free_session_memory(scd_session *s)
     if (s->attn_plan) attention_session_release(s);
 }
 
-// A bounded device-side wait that gave up leaves a non-zero error word.
+// A bounded device-side wait that gave up leaves a non-zero error word (sticky until the next prefill:
+// the GEMM kernels skip their output operation while it is set).
 int check_device_health(scd_session *s, cudaStream_t st)
 {
     int word = 0;
     int rc = gemm_error_word(s, &word, st);
     if (rc != SCD_OK) return rc;
-    SCD_REQUIRE(word == 0, SCD_ERR_TIMEOUT, "a bounded wait inside the GEMM kernel gave up (role %d)", word);
+    static const char *const who[] = {"", "GEMM: producer waiting for a free ring slot", "GEMM: MMA issuer waiting for operands",
+                                      "GEMM: epilogue waiting for the accumulator", "attention: waiting for a free ring slot",
+                                      "attention: waiting for a K/V tile", "attention: shared memory base not 1024-byte aligned"};
+    SCD_REQUIRE(word == 0, SCD_ERR_TIMEOUT, "a bounded device-side wait gave up (%s, code %d); prefill the session again",
+                word > 0 && word < 7 ? who[word] : "unknown", word);
     return SCD_OK;
 }
 
@@ -337,6 +342,7 @@ int scd_prefill(scd_session_t *s, const int32_t *prompt_ids, int32_t P, int32_t 
     s->n_new = n_new;
     s->prefilled = false;
     drop_step_graph(s);                                  // the prompt length is baked into the captured launches
+    if (s->gemm_ws) SCD_CUDA_TRY(cudaMemsetAsync(s->gemm_ws, 0, s->gemm_ws_bytes, st));   // a fresh start clears the error word
     // token records: conditional prompts -> tokens, unconditional prompts -> tokens_u
     std::memcpy(s->host_pinned, prompt_ids, (size_t)s->Q * P * sizeof(int));
     SCD_CUDA_TRY(cudaMemcpy2DAsync(s->tokens, (size_t)c.max_seq * sizeof(int), s->host_pinned,

@@ -23,6 +23,12 @@ int cuda_fail(cudaError_t e, const char *what)
     return SCD_ERR_CUDA;
 }
 
+int current_device(int *device)
+{
+    SCD_CUDA_TRY(cudaGetDevice(device));
+    return SCD_OK;
+}
+
 int validate_decode_config(const scd_decode_config_t *cfg, int V)
 {
     SCD_REQUIRE(cfg != nullptr, SCD_ERR_ARG, "decode config is NULL");
@@ -102,7 +108,8 @@ __global__ void noise_kernel(unsigned long long seed, unsigned stream, unsigned 
 // name is only a host-side stand-in: the device address is looked up once per device.
 #define SCD_NOALLOC_SCRATCH_BYTES (16u << 20)
 static __device__ __align__(256) unsigned char g_noalloc_scratch[SCD_NOALLOC_SCRATCH_BYTES];
-static void *g_noalloc_scratch_addr[64];      // per device ordinal; 0 = not looked up yet
+static void *g_noalloc_scratch_addr[DeviceOnce::kSlots];      // per device ordinal, filled under g_noalloc_once
+static DeviceOnce g_noalloc_once;
 
 }  // namespace scd
 
@@ -187,6 +194,24 @@ int scd_noise_u24(uint64_t seed, uint32_t noise_stream, uint32_t batch, const in
     return SCD_OK;
 }
 
+int scd_selftest_device_once(void)
+{
+    // host-only: the per-device bookkeeping behind the kernels' one-time set-up
+    DeviceOnce once;
+    int runs = 0;
+    auto ok = [&]() -> int { ++runs; return SCD_OK; };
+    auto bad = [&]() -> int { ++runs; return SCD_ERR_CUDA; };
+    if (once.run(0, ok) != SCD_OK || runs != 1) return 1;
+    if (once.run(0, ok) != SCD_OK || runs != 1) return 2;          // second use of device 0: skipped
+    if (once.run(1, ok) != SCD_OK || runs != 2) return 3;          // another device: runs again
+    if (once.run(2, bad) != SCD_ERR_CUDA || runs != 3) return 4;   // a failed set-up ...
+    if (once.run(2, ok) != SCD_OK || runs != 4) return 5;          // ... is tried again
+    if (once.run(2, ok) != SCD_OK || runs != 4) return 6;
+    if (once.run(DeviceOnce::kSlots + 3, ok) != SCD_OK || once.run(DeviceOnce::kSlots + 3, ok) != SCD_OK || runs != 6)
+        return 7;                                                  // beyond the table: every time
+    return 0;
+}
+
 int64_t scd_verify_noalloc_max_bytes(void) { return (int64_t)SCD_NOALLOC_SCRATCH_BYTES; }
 
 int scd_verify_noalloc(const scd_decode_config_t *cfg, int32_t V, const float *p_logits,
@@ -202,15 +227,19 @@ int scd_verify_noalloc(const scd_decode_config_t *cfg, int32_t V, const float *p
                 "buffer holds %u; use scd_verify with a caller-allocated workspace", cfg->batch,
                 cfg->window_L, V, (long long)need, SCD_NOALLOC_SCRATCH_BYTES);
     int dev = 0;
-    SCD_CUDA_TRY(cudaGetDevice(&dev));
-    SCD_REQUIRE(dev >= 0 && dev < 64, SCD_ERR_UNSUPPORTED, "scd_verify_noalloc: device ordinal %d", dev);
-    if (!g_noalloc_scratch_addr[dev]) {
-        // first call on this device: resolve the device address of the built-in buffer
+    rc = current_device(&dev);
+    if (rc != SCD_OK) return rc;
+    SCD_REQUIRE(dev >= 0 && dev < DeviceOnce::kSlots, SCD_ERR_UNSUPPORTED, "scd_verify_noalloc: device ordinal %d", dev);
+    // first call on this device: resolve the device address of the built-in buffer (this is also the
+    // moment the CUDA runtime loads this module on the device and gives the array its memory)
+    rc = g_noalloc_once.run(dev, [&]() -> int {
         void *ptr = nullptr;
         SCD_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
         SCD_REQUIRE(ptr != nullptr, SCD_ERR_CUDA, "scd_verify_noalloc: no device address for the scratch buffer");
         g_noalloc_scratch_addr[dev] = ptr;
-    }
+        return SCD_OK;
+    });
+    if (rc != SCD_OK) return rc;
     // scd_verify zeroes the part of the workspace that must start at zero (the per-sequence
     // tickets) on `stream` before the kernel; everything else is written before it is read
     return scd_verify(cfg, V, p_logits, q_logits, draft_ids, positions, iteration, n_commit, committed_ids,

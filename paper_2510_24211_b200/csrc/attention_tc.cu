@@ -706,15 +706,19 @@ int attention_tc(scd_session *s, int layer, int Mq, int pos_override, cudaStream
     p.stages = stages;
     const size_t smem = q_bytes + (size_t)stages * stage_bytes;
     SCD_REQUIRE(smem <= 227 * 1024 - 4096, SCD_ERR_SHAPE, "attention needs %zu bytes of shared memory", smem);
-    static bool configured = false;
-    if (!configured) {
+    static DeviceOnce once;
+    int dev = 0;
+    int rc = current_device(&dev);
+    if (rc != SCD_OK) return rc;
+    rc = once.run(dev, [&]() -> int {
         const int lim = 227 * 1024 - 4096;
         SCD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim));
         SCD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim));
         SCD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim));
         SCD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim));
-        configured = true;
-    }
+        return SCD_OK;
+    });
+    if (rc != SCD_OK) return rc;
     // two warps per query tile once the context is known to be long (see attention_tc_wide)
     const bool wide = pos_override < 0 && attention_tc_wide(s, Mq);
     cudaLaunchConfig_t cfg;

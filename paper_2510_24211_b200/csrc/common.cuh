@@ -5,8 +5,9 @@
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
+#include <mutex>
 
-#include "../../include/scd.h"
+#include "../../include/scd_hooks.h"
 
 namespace scd {
 
@@ -17,6 +18,26 @@ void set_last_error(const char *fmt, ...);
 int cuda_fail(cudaError_t e, const char *what);
 // Kernels enqueued by this process so far: every launch site counts itself.
 void count_launches(long long n);
+
+// Set-up that a CUDA device needs once (a kernel's shared-memory opt-in is a per-device attribute, the
+// address of a __device__ array differs per device): `done` remembers the ordinals it has run on, the
+// lock keeps a second host thread from launching before the first has finished the set-up.
+struct DeviceOnce {
+    static constexpr int kSlots = 64;
+    std::mutex lock;
+    bool done[kSlots] = {};
+    // Runs setup() unless it already succeeded on `device`; ordinals beyond the table run it every time.
+    template <class F>
+    int run(int device, F setup)
+    {
+        std::lock_guard<std::mutex> g(lock);
+        if (device >= 0 && device < kSlots && done[device]) return SCD_OK;
+        const int rc = setup();
+        if (rc == SCD_OK && device >= 0 && device < kSlots) done[device] = true;
+        return rc;
+    }
+};
+int current_device(int *device);    // cudaGetDevice as a status code
 
 #define SCD_CUDA_TRY(expr)                                                     \
     do {                                                                       \

@@ -624,9 +624,8 @@ struct GemmPlan {                    // per model: weight-side tensor maps, buil
     std::map<std::tuple<const void *, int, int, int>, CUtensorMap> wmaps;   // (matrix, rows, K, box rows)
     int sm_count;
     int kind_splits[GEMM_KINDS];     // K slices per GEMM kind chosen by gemm_set_kind_splits (0: the rule)
+    int forced_splits, forced_stages; // scd_model_gemm_tune (0: the rule)
 };
-
-int g_forced_splits = 0, g_forced_stages = 0;
 
 inline int round16(int m) { return std::max(16, (m + 15) & ~15); }
 
@@ -649,12 +648,12 @@ int tiles_for(const Segment *segs, int n_seg, bool pair, int h)
 // tile is re-read per weight tile), and a CTA should stream at most ~32 K blocks. So: full-height
 // tiles and the smallest C that gives every SM two CTAs.
 void choose_shape(const Segment *segs, int n_seg, bool pair, int k_blocks, int sm_count, int *C_out, int *h_out,
-                  int *tiles_out, int tuned = 0)
+                  int *tiles_out, int tuned = 0, int forced = 0)
 {
     const int h = pair ? TILE_N / 2 : TILE_N;
     const int tiles = tiles_for(segs, n_seg, pair, h);
     int C;
-    if (g_forced_splits > 0) C = g_forced_splits;
+    if (forced > 0) C = forced;
     else if (tuned > 0) C = tuned;
     else {
         C = (k_blocks + 31) / 32;
@@ -668,11 +667,11 @@ void choose_shape(const Segment *segs, int n_seg, bool pair, int k_blocks, int s
 // Ring slots: about 72 KB per CTA so that three CTAs share an SM - or about 100 KB when the grid has
 // at most two CTAs per SM anyway (measured: the deeper ring then wins a few percent) - and never
 // less than the partial-tile staging.
-int choose_stages(int nbox, int k_blocks_per_cta, bool two_per_sm)
+int choose_stages(int nbox, int k_blocks_per_cta, bool two_per_sm, int forced = 0)
 {
     const int stage_bytes = (int)stage_bytes_of(nbox);
     int st = std::max(2, ((two_per_sm ? 100 : 73) * 1024) / stage_bytes);
-    if (g_forced_stages > 0) st = g_forced_stages;
+    if (forced > 0) st = forced;
     st = std::min(st, (int)((SMEM_LIMIT - 1024) / stage_bytes));
     st = std::min(st, MAX_STAGES);
     st = std::min(st, std::max(2, k_blocks_per_cta));
@@ -687,11 +686,15 @@ int launch(GemmParams &p, int tiles, cudaStream_t st)
     size_t smem = ring + 5 * rows_per_cta * sizeof(float) + 1024;
     SCD_REQUIRE(smem <= SMEM_LIMIT, SCD_ERR_SHAPE, "GEMM needs %zu bytes of shared memory", smem);
     SCD_REQUIRE(p.M <= MAX_ROWS, SCD_ERR_SHAPE, "GEMM carries at most %d window rows", MAX_ROWS);
-    static bool configured = false;
-    if (!configured) {
+    static DeviceOnce once;
+    int dev = 0;
+    int rc = current_device(&dev);
+    if (rc != SCD_OK) return rc;
+    rc = once.run(dev, [&]() -> int {
         SCD_CUDA_TRY(cudaFuncSetAttribute(gemm_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT));
-        configured = true;
-    }
+        return SCD_OK;
+    });
+    if (rc != SCD_OK) return rc;
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)(tiles * p.k_splits), 1, 1);
@@ -761,7 +764,7 @@ int run_gemm(scd_session *s, int kind, const Segment *segs, int n_seg, int epi, 
     p.k_blocks = K / BLOCK_K;
     int tiles = 0;
     choose_shape(segs, n_seg, pair, p.k_blocks, plan->sm_count, &p.k_splits, &p.tile_rows, &tiles,
-                 plan->kind_splits[kind]);
+                 plan->kind_splits[kind], plan->forced_splits);
     int t0 = 0;
     for (int i = 0; i < n_seg; ++i) {
         int rc = w_map(plan, segs[i], p.tile_rows, &p.tmap_w[i]);
@@ -775,7 +778,8 @@ int run_gemm(scd_session *s, int kind, const Segment *segs, int n_seg, int epi, 
     p.n_seg = pair ? 1 : n_seg;
     p.M = rows;
     p.nbox = round16(rows);
-    p.stages = choose_stages(p.nbox, (p.k_blocks + p.k_splits - 1) / p.k_splits, tiles * p.k_splits <= 2 * plan->sm_count);
+    p.stages = choose_stages(p.nbox, (p.k_blocks + p.k_splits - 1) / p.k_splits, tiles * p.k_splits <= 2 * plan->sm_count,
+                             plan->forced_stages);
     p.epi = epi;
     p.out = out;
     p.ldo = ldo;
@@ -805,6 +809,7 @@ int gemm_plan_create(scd_model *m)
     cudaGetDevice(&dev);
     plan->sm_count = 148;
     for (int k = 0; k < GEMM_KINDS; ++k) plan->kind_splits[k] = 0;
+    plan->forced_splits = plan->forced_stages = 0;
     if (cudaDeviceGetAttribute(&plan->sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
         delete plan;
         return cuda_fail(cudaGetLastError(), "cudaDeviceGetAttribute");
@@ -917,19 +922,26 @@ int64_t scd_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K)
     return 256;                                           // the device error word
 }
 
-int scd_gemm_tune(int32_t k_splits, int32_t stages)
+int scd_model_gemm_tune(scd_model_t *m, int32_t k_splits, int32_t stages)
 {
-    g_forced_splits = k_splits;
-    g_forced_stages = stages;
+    SCD_REQUIRE(m, SCD_ERR_ARG, "scd_model_gemm_tune: NULL model");
+    SCD_REQUIRE(k_splits >= 0 && k_splits <= MAX_CLUSTER && stages >= 0 && stages <= MAX_STAGES, SCD_ERR_ARG,
+                "scd_model_gemm_tune: k_splits %d (0..%d), stages %d (0..%d)", k_splits, MAX_CLUSTER, stages, MAX_STAGES);
+    GemmPlan *plan = (GemmPlan *)m->gemm_plan;
+    if (!plan) return SCD_OK;                             // fp32 model: no tcgen05 GEMMs to shape
+    plan->forced_splits = k_splits;
+    plan->forced_stages = stages;
     return SCD_OK;
 }
 
-int scd_gemm_bf16(const void *x, const void *w, float *y, int32_t M, int32_t N, int32_t K, void *workspace,
-                  void *stream)
+int scd_gemm_bf16_shaped(const void *x, const void *w, float *y, int32_t M, int32_t N, int32_t K, int32_t k_splits,
+                         int32_t stages, void *workspace, void *stream)
 {
     SCD_REQUIRE(x && w && y && workspace, SCD_ERR_ARG, "scd_gemm_bf16: NULL argument");
     SCD_REQUIRE(M >= 1 && M <= 256 && N >= 1 && N % 8 == 0 && K >= BLOCK_K && K % BLOCK_K == 0, SCD_ERR_SHAPE,
                 "scd_gemm_bf16: M %d (1..256), N %d (multiple of 8), K %d (multiple of 64)", M, N, K);
+    SCD_REQUIRE(k_splits >= 0 && k_splits <= MAX_CLUSTER && stages >= 0 && stages <= MAX_STAGES, SCD_ERR_ARG,
+                "scd_gemm_bf16: k_splits %d (0..%d), stages %d (0..%d)", k_splits, MAX_CLUSTER, stages, MAX_STAGES);
     SCD_REQUIRE((((uintptr_t)x | (uintptr_t)w | (uintptr_t)workspace) & 15) == 0, SCD_ERR_ARG,
                 "scd_gemm_bf16: pointers must be 16-byte aligned");
     int dev = 0, sms = 148;
@@ -940,7 +952,7 @@ int scd_gemm_bf16(const void *x, const void *w, float *y, int32_t M, int32_t N, 
     p.k_blocks = K / BLOCK_K;
     const Segment seg = {w, N, K, 0, N, 0};
     int tiles = 0;
-    choose_shape(&seg, 1, false, p.k_blocks, sms, &p.k_splits, &p.tile_rows, &tiles);
+    choose_shape(&seg, 1, false, p.k_blocks, sms, &p.k_splits, &p.tile_rows, &tiles, 0, k_splits);
     int rc = make_map(&p.tmap_w[0], w, (uint64_t)N, (uint64_t)K, (uint32_t)p.tile_rows);
     if (rc != SCD_OK) return rc;
     p.nbox = round16(M);
@@ -949,12 +961,18 @@ int scd_gemm_bf16(const void *x, const void *w, float *y, int32_t M, int32_t N, 
     if (rc != SCD_OK) return rc;
     p.seg_tile0[0] = 0; p.seg_tile0[1] = tiles; p.seg_row0[0] = 0; p.seg_nout[0] = N; p.seg_col0[0] = 0; p.n_seg = 1;
     p.M = M;
-    p.stages = choose_stages(p.nbox, (p.k_blocks + p.k_splits - 1) / p.k_splits, tiles * p.k_splits <= 2 * sms);
+    p.stages = choose_stages(p.nbox, (p.k_blocks + p.k_splits - 1) / p.k_splits, tiles * p.k_splits <= 2 * sms, stages);
     p.epi = EPI_F32;
     p.out = y;
     p.ldo = N;
     p.err = (int *)workspace;                             // must be zero on entry; stays zero unless a wait gave up
     return launch(p, tiles, (cudaStream_t)stream);
+}
+
+int scd_gemm_bf16(const void *x, const void *w, float *y, int32_t M, int32_t N, int32_t K, void *workspace,
+                  void *stream)
+{
+    return scd_gemm_bf16_shaped(x, w, y, M, N, K, 0, 0, workspace, stream);
 }
 
 }  // extern "C"

@@ -682,9 +682,10 @@ __global__ void __launch_bounds__(VT, 1) verify_kernel(const VerifyParams p, int
                 }
                 const unsigned Ua = noise_u24(p.seed, NOISE_ACCEPT, (unsigned)b, pos, w.t, 0);
                 // u <= min(1, p(X)/q(X)) with u = (Ua+1)/2^24  <=>  (Ua+1) Wq[X] Zp <= Wp[X] Zq 2^24
+                // (a draft without mass under p - possible only when X was not drawn from q - is rejected)
                 const u128 lhs = (u128)(Ua + 1u) * WqX * Zp;
                 const u128 rhs = ((u128)WpX * Zq) << 24;
-                sm.flag = lhs <= rhs ? 1 : 0;
+                sm.flag = (WpX != 0u && lhs <= rhs) ? 1 : 0;
             }
             __syncthreads();
             accept = sm.flag;
@@ -848,11 +849,15 @@ int launch_verify(const VerifyParams &p, cudaStream_t stream)
     if ((size_t)n * 8 <= budget) { stage_cap = n; stage_q = 1; }
     else if ((size_t)n * 4 <= budget) { stage_cap = n; }
     const size_t smem = (size_t)stage_cap * 4 * (stage_q ? 2 : 1);
-    static size_t configured = 0;
-    if (smem > configured) {
+    static DeviceOnce once;
+    int dev = 0;
+    int rc = current_device(&dev);
+    if (rc != SCD_OK) return rc;
+    rc = once.run(dev, [&]() -> int {
         SCD_CUDA_TRY(cudaFuncSetAttribute(verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
-        configured = budget;
-    }
+        return SCD_OK;
+    });
+    if (rc != SCD_OK) return rc;
     verify_kernel<<<grid, VT, smem, stream>>>(p, stage_cap, stage_q);
     SCD_CUDA_TRY(cudaGetLastError());
     return SCD_OK;

@@ -1,5 +1,5 @@
 """The C-ABI boundary without a GPU: the shared library loads, exports every function that
-include/scd.h declares (and the binding lists the same names), the ctypes structures have the
+include/*.h declare (and the binding lists the same names), the ctypes structures have the
 layout the C compiler gives the header's structs, and the calls that need no device answer."""
 import ctypes as C
 import os
@@ -12,12 +12,13 @@ import pytest
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 sys.path.insert(0, ROOT)
 HEADER = os.path.join(ROOT, "include", "scd.h")
+HEADERS = [HEADER, os.path.join(ROOT, "include", "scd_hooks.h")]
 
 from paper_2510_24211_b200 import binding as scd  # noqa: E402
 
 
 def _declared():
-    text = open(HEADER).read()
+    text = "".join(open(h).read() for h in HEADERS)
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)          # comments mention function names too
     return re.findall(r"^\s*(?:int|int64_t|const char \*)\s*\*?\s*(scd_\w+)\s*\(", text, flags=re.M)
 
@@ -27,7 +28,7 @@ def test_library_exports_every_declared_function():
     assert len(names) >= 20 and len(set(names)) == len(names)
     lib = C.CDLL(scd.LIB_PATH)
     for n in names:
-        assert hasattr(lib, n), f"{n} is declared in scd.h but not exported"
+        assert hasattr(lib, n), f"{n} is declared in include/ but not exported"
     assert set(names) == set(scd.EXPORTS)
 
 
@@ -61,6 +62,7 @@ def test_calls_that_need_no_device():
     texts = {code: lib.scd_strerror(code).decode() for code in range(-8, 1)}
     assert texts[0] and len(set(texts.values())) >= 8             # one text per status code
     assert scd.scd_kernel_launches() >= 0
+    assert scd.scd_selftest_device_once() == 0                    # per-device set-up bookkeeping (host only)
     # argument checks run on the host, before any CUDA call
     bad = scd.decode_config(batch=0, window_L=4, allowed_hi=10)
     assert lib.scd_verify_workspace_bytes(C.byref(bad), 10) < 0

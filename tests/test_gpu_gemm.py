@@ -9,19 +9,19 @@ from paper_2510_24211_b200 import binding as scd
 pytestmark = pytest.mark.gpu
 
 
-def _check(M, N, K, seed=0):
+def _check(M, N, K, seed=0, k_splits=0, stages=0):
     g = torch.Generator(device="cuda")
     g.manual_seed(seed)
     x = torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16)
     w = (torch.randn(N, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16)
-    y = scd.scd_gemm_bf16(x, w)
+    y = scd.scd_gemm_bf16(x, w, k_splits=k_splits, stages=stages)
     torch.cuda.synchronize()
     ref = x.double() @ w.double().T
     scale = (x.double().abs() @ w.double().abs().T).max().item()
     err = (y.double() - ref).abs().max().item()
     assert err <= 2e-6 * scale, (M, N, K, err, scale)
     # deterministic: split-K partials are added in a fixed order
-    y2 = scd.scd_gemm_bf16(x, w)
+    y2 = scd.scd_gemm_bf16(x, w, k_splits=k_splits, stages=stages)
     assert torch.equal(y, y2)
 
 
@@ -30,18 +30,13 @@ def _check(M, N, K, seed=0):
     (256, 512, 704), (17, 4096, 11008), (2, 16384, 1280), (64, 4096, 4096), (100, 8, 64),
 ])
 def test_gemm_matches_fp64_matmul(M, N, K):
-    scd.scd_gemm_tune(0, 0)
     _check(M, N, K)
 
 
 @pytest.mark.parametrize("splits,stages", [(1, 2), (2, 3), (7, 4), (8, 2), (3, 12), (5, 3)])
 def test_gemm_forced_slices_and_stages(splits, stages):
-    try:
-        scd.scd_gemm_tune(splits, stages)
-        _check(64, 1024, 2048, seed=splits)
-        _check(48, 384, 512, seed=stages)
-    finally:
-        scd.scd_gemm_tune(0, 0)
+    _check(64, 1024, 2048, seed=splits, k_splits=splits, stages=stages)
+    _check(48, 384, 512, seed=stages, k_splits=splits, stages=stages)
 
 
 def test_gemm_rejects_bad_shapes():

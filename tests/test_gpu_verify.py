@@ -163,3 +163,22 @@ def test_verify_rejects_bad_arguments():
     # the context is still usable
     scd.scd_verify(cfg, p, None, d, pos, 0)
     torch.cuda.synchronize()
+
+
+def test_verify_draft_without_mass_is_rejected():
+    """Drafts that have no mass under p (outside its top-k; some outside q's as well, which X ~ q rules
+    out but a caller can hand in): never accepted, the row's output comes from the residual."""
+    B, L, V, top_k, seed = 2, 6, 2000, 20, 51
+    p, q = synth.verify_logits(seed, 0, B, L, V, device="cuda")
+    drafts = torch.argmin(p[0] + q, dim=-1).to(torch.int32)          # far below both thresholds
+    drafts[0, 1] = torch.argmax(q[0, 1]).to(torch.int32)              # one ordinary row in between
+    positions = torch.tensor([300, 900], dtype=torch.int64, device="cuda")
+    cfg = scd.decode_config(mode=scd.SCD_MODE_SCD_MC, batch=B, window_L=L, top_k=top_k, seed=seed, allowed_hi=V)
+    got = [t.cpu().numpy() for t in scd.scd_verify(cfg, p, q, drafts, positions, 3)]
+    want = oracle_verify("scd", p.cpu().numpy(), q.cpu().numpy(), drafts.cpu().numpy(), positions.cpu().numpy(),
+                         3, seed, 1.0, top_k)
+    assert np.array_equal(got[0], want["n_commit"]) and np.array_equal(got[3], want["flags"])
+    assert np.array_equal(got[2], want["next_drafts"])
+    assert (got[3][:, 0] == 0).all() and (got[0] == 1).all()         # row 0 of both sequences rejects
+    for b in range(B):
+        assert got[1][b, 0] == want["committed"][b, 0] and got[1][b, 0] != drafts[b, 0].item()

@@ -445,3 +445,17 @@ def test_alpha_coin_rate_and_coupling_cost(alpha):
     tvd = 0.5 * np.abs(P - Q).sum()
     cost = alpha * (1.0 - tvd) + (1.0 - alpha) * float((P * Q).sum())
     assert abs(n_same / n_rows - cost) <= 5 * math.sqrt(cost * (1 - cost) / n_rows)
+
+
+def test_mrs_never_emits_an_id_without_mass():
+    # Algorithm 1 returns a sample of p (Prop. 2.1): a draft outside the support of p is rejected even
+    # when it is outside the support of q as well (a caller's mistake, since X ~ q), and the output
+    # then comes from norm(max(0, p - q)), whose support lies inside that of p.
+    Wp = np.array([0, 5, 0, 3, 9, 0], dtype=np.uint32)
+    Wq = np.array([0, 2, 7, 0, 4, 1], dtype=np.uint32)
+    Zp, Zq = int(Wp.sum()), int(Wq.sum())
+    for X in (0, 2, 5):                                   # p(X) = 0; q(X) = 0 for X = 0
+        for Ua in (0, 1, N24 // 2, N24 - 1):
+            for Ur in (0, N24 // 3, N24 - 1):
+                k, Y = oracle.mrs(Wp, Zp, Wq, Zq, X, Ua, Ur)
+                assert k == 0 and Wp[Y] > 0

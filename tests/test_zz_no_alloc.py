@@ -11,9 +11,11 @@ large for the buffer is refused without launching anything.
 Collected last on purpose (file name), so that a run stopping at the first failure has already
 run every other test. It needs no state from other tests: every tensor is created here, before
 the calls, and the calls themselves allocate nothing."""
+import numpy as np
 import pytest
 import torch
 
+from helpers import oracle_verify
 from paper_2510_24211_b200 import binding as scd
 from paper_2510_24211_b200 import synth
 
@@ -55,11 +57,25 @@ def test_noalloc_matches_scd_verify_twice_in_a_row():
         for b in range(B):
             a = int(want[0][b])
             assert torch.equal(got[1][b, :a], want[1][b, :a])     # committed ids (first a are defined)
-        # same call again on the same inputs: same answer (nothing left over changes it)
+        # same call again on the same inputs: same answer (nothing left over changes it), and - the
+        # first call on this device being behind us - no device memory is taken by the call
         out2 = _outputs(B, L)
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
         got2 = scd.scd_verify_noalloc(cfg, p, q, drafts, positions, it, out2)
         torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        assert free_after == free_before
         assert torch.equal(got2[0], want[0]) and torch.equal(got2[2], want[2]) and torch.equal(got2[3], want[3])
+        # and against the CPU oracle, like every other verify test
+        ref = oracle_verify("scd", p.cpu().numpy(), q.cpu().numpy(), drafts.cpu().numpy(), positions.cpu().numpy(),
+                            it, 5, 1.0, top_k, lam)
+        assert np.array_equal(got2[0].cpu().numpy(), ref["n_commit"])
+        assert np.array_equal(got2[3].cpu().numpy(), ref["flags"])
+        assert np.array_equal(got2[2].cpu().numpy(), ref["next_drafts"])
+        for b in range(B):
+            a = int(ref["n_commit"][b])
+            assert np.array_equal(got2[1][b, :a].cpu().numpy(), ref["committed"][b, :a])
 
 
 def test_noalloc_refuses_what_does_not_fit():
