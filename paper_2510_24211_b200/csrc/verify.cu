@@ -44,16 +44,6 @@ struct Smem {
     int flag;
 };
 
-__device__ __forceinline__ void allowed_range(const VerifyParams &p, long long pos, int &lo, int &hi)
-{
-    const long long g = pos - p.prompt_len;
-    if (p.row_period > 0 && g >= 0 && (g % p.row_period) == p.row_period - 1) {
-        lo = p.eol_id; hi = p.eol_id + 1;
-    } else {
-        lo = p.allowed_lo; hi = p.allowed_hi;
-    }
-}
-
 // Post-processed logit of id v of a stored row; raw draft logits still need the temperature.
 struct XRow {
     const float *row;      // global row (off = 0) or its copy in shared memory (off = first allowed id)
@@ -329,17 +319,6 @@ __device__ unsigned nucleus_threshold(const F &weight, int lo, int hi, unsigned 
     return prefix;
 }
 
-// w * z for a 32-bit weight and a 64-bit normaliser as a 128-bit value, from two 32 x 32 -> 64
-// products (the general 128-bit multiply costs several times more).
-__device__ __forceinline__ u128 mul_32x64(unsigned w, unsigned long long z)
-{
-    const unsigned long long p0 = (unsigned long long)w * (unsigned)z;
-    const unsigned long long p1 = (unsigned long long)w * (unsigned)(z >> 32);
-    const unsigned long long lo = p0 + (p1 << 32);
-    const unsigned long long hi = (p1 >> 32) + (lo < p0 ? 1ull : 0ull);
-    return ((u128)hi << 64) | lo;
-}
-
 // Inverse-CDF search: smallest id v in [lo, hi) with sum_{v' <= v} f(v') > (U * total) >> 24,
 // ids in increasing order. Warps own contiguous id ranges; the warp whose range holds the
 // target walks it 32 ids at a time. Returns -1 when the total is zero.
@@ -395,16 +374,6 @@ __device__ int block_search(const F &f, int lo, int hi, unsigned U, Smem &sm)
     return res;
 }
 
-// Draft of a row that enters the window: X ~ uniform over the allowed ids of its position
-// (the initialisation of Algorithm 6: "p <- Random(); X ~ p").
-__device__ __forceinline__ int fresh_draft(const VerifyParams &p, int b, long long pos, unsigned first_iter)
-{
-    int lo, hi;
-    allowed_range(p, pos, lo, hi);
-    const unsigned U = noise_u24(p.seed, NOISE_INIT, (unsigned)b, pos, first_iter, 0);
-    return lo + (int)(((unsigned long long)U * (unsigned long long)(hi - lo)) >> 24);
-}
-
 // ---- Gumbel race (Algorithm 4, in the exponential-race form of its proof) ----------------------
 // Candidate v finishes at E_v / W_v, E_v = -log2 u_v in fixed point; the earliest wins. Times are
 // compared by cross-multiplication in 128 bits and ties go to the smaller id: a strict total
@@ -447,35 +416,6 @@ __device__ int block_race(const F &weight, int lo, int hi, const VerifyParams &p
     }
     __syncthreads();
     return r.v;
-}
-
-struct WindowState {
-    long long pos0;
-    int Lw, shift, prev_lw, parity;
-    unsigned t;
-};
-
-__device__ __forceinline__ WindowState load_state(const VerifyParams &p, int b)
-{
-    WindowState w;
-    if (p.n_known) {
-        const int n = p.n_known[b];
-        w.pos0 = n;
-        w.Lw = max(0, min(p.L, p.n_total[b] - n));
-        w.t = p.iter[b];
-        w.parity = (int)(w.t & 1u);
-        w.shift = p.shift[b];
-        w.prev_lw = p.prev_lw[b];
-    } else {
-        w.pos0 = p.positions[b];
-        w.Lw = p.L;
-        w.t = (unsigned)p.iteration;
-        w.parity = 0;
-        w.shift = 0;
-        w.prev_lw = p.q_present ? p.L : 0;
-    }
-    if (p.mode == SCD_MODE_AR) w.Lw = min(w.Lw, 1);
-    return w;
 }
 
 // Rows are staged in shared memory when they fit (stage_cap floats per row; stage_q: a second
@@ -841,6 +781,9 @@ __global__ void init_window_kernel(const VerifyParams p)
 
 int launch_verify(const VerifyParams &p, cudaStream_t stream)
 {
+    // a cluster per row wherever it applies; this kernel keeps the Gumbel race, the nucleus truncation
+    // and rows too long for a cluster's registers
+    if (verify_cluster_supported(p)) return launch_verify_cluster(p, stream);
     dim3 grid((unsigned)p.L, (unsigned)p.B);
     // shared-memory staging: both rows if they fit, else the target row alone, else none
     const int n = p.allowed_hi - p.allowed_lo;

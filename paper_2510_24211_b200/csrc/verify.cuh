@@ -65,7 +65,73 @@ struct VerifyParams {
     VerifyStatsDev *dev_stats;    // session counters (or NULL)
 };
 
+// ---- device helpers shared by the two verify kernels -----------------------------------------------
+// ids a position may take: the allowed range, or the single end-of-row id at forced positions
+__device__ __forceinline__ void allowed_range(const VerifyParams &p, long long pos, int &lo, int &hi)
+{
+    const long long g = pos - p.prompt_len;
+    if (p.row_period > 0 && g >= 0 && (g % p.row_period) == p.row_period - 1) {
+        lo = p.eol_id; hi = p.eol_id + 1;
+    } else {
+        lo = p.allowed_lo; hi = p.allowed_hi;
+    }
+}
+
+// w * z for a 32-bit weight and a 64-bit normaliser as a 128-bit value, from two 32 x 32 -> 64
+// products (the general 128-bit multiply costs several times more).
+__device__ __forceinline__ u128 mul_32x64(unsigned w, unsigned long long z)
+{
+    const unsigned long long p0 = (unsigned long long)w * (unsigned)z;
+    const unsigned long long p1 = (unsigned long long)w * (unsigned)(z >> 32);
+    const unsigned long long lo = p0 + (p1 << 32);
+    const unsigned long long hi = (p1 >> 32) + (lo < p0 ? 1ull : 0ull);
+    return ((u128)hi << 64) | lo;
+}
+
+// Draft of a row that enters the window: X ~ uniform over the allowed ids of its position
+// (the initialisation of Algorithm 6: "p <- Random(); X ~ p").
+__device__ __forceinline__ int fresh_draft(const VerifyParams &p, int b, long long pos, unsigned first_iter)
+{
+    int lo, hi;
+    allowed_range(p, pos, lo, hi);
+    const unsigned U = noise_u24(p.seed, NOISE_INIT, (unsigned)b, pos, first_iter, 0);
+    return lo + (int)(((unsigned long long)U * (unsigned long long)(hi - lo)) >> 24);
+}
+
+// Window of one sequence at this iteration (session: device-resident counters; stand-alone: arguments)
+struct WindowState {
+    long long pos0;
+    int Lw, shift, prev_lw, parity;
+    unsigned t;
+};
+
+__device__ __forceinline__ WindowState load_state(const VerifyParams &p, int b)
+{
+    WindowState w;
+    if (p.n_known) {
+        const int n = p.n_known[b];
+        w.pos0 = n;
+        w.Lw = max(0, min(p.L, p.n_total[b] - n));
+        w.t = p.iter[b];
+        w.parity = (int)(w.t & 1u);
+        w.shift = p.shift[b];
+        w.prev_lw = p.prev_lw[b];
+    } else {
+        w.pos0 = p.positions[b];
+        w.Lw = p.L;
+        w.t = (unsigned)p.iteration;
+        w.parity = 0;
+        w.shift = 0;
+        w.prev_lw = p.q_present ? p.L : 0;
+    }
+    if (p.mode == SCD_MODE_AR) w.Lw = min(w.Lw, 1);
+    return w;
+}
+
 int launch_verify(const VerifyParams &p, cudaStream_t stream);
+// the kernel that gives every window row a thread-block cluster (verify_cluster.cu)
+bool verify_cluster_supported(const VerifyParams &p);
+int launch_verify_cluster(const VerifyParams &p, cudaStream_t stream);
 int launch_init_window(const VerifyParams &p, cudaStream_t stream);
 
 }  // namespace scd
