@@ -288,11 +288,13 @@ int scd_session_create(scd_model_t *m, const scd_decode_config_t *cfg, scd_sessi
     TRY_ALLOC(dev_alloc(&s->stats[1], wrows));
     TRY_ALLOC(dev_alloc(&s->dev_stats, 1));
     TRY_ALLOC(dev_alloc(&s->h, rows * d));
-    { char *p; TRY_ALLOC(dev_alloc(&p, rows * d * es)); s->xn = p; }
-    { char *p; TRY_ALLOC(dev_alloc(&p, rows * (dq + 2 * dkv) * es)); s->qkv = p; }
-    { char *p; TRY_ALLOC(dev_alloc(&p, rows * dq * es)); s->att = p; }
+    // bf16 sessions: GEMM inputs (xn, att, act) in two bf16 planes [2][rows][K], projections (qkv) in fp32
+    const size_t wide = c.dtype == SCD_BF16 ? 2 : 1;
+    { char *p; TRY_ALLOC(dev_alloc(&p, wide * rows * d * es)); s->xn = p; }
+    { char *p; TRY_ALLOC(dev_alloc(&p, wide * rows * (dq + 2 * dkv) * es)); s->qkv = p; }
+    { char *p; TRY_ALLOC(dev_alloc(&p, wide * rows * dq * es)); s->att = p; }
     { char *p; TRY_ALLOC(dev_alloc(&p, rows * 2 * F * es)); s->gu = p; }
-    { char *p; TRY_ALLOC(dev_alloc(&p, rows * F * es)); s->act = p; }
+    { char *p; TRY_ALLOC(dev_alloc(&p, wide * rows * F * es)); s->act = p; }
     s->ss_parts_cap = c.dtype == SCD_BF16 && m->gemm_plan ? gemm_norm_parts_cap(s) : 1;
     TRY_ALLOC(dev_alloc(&s->ss, (size_t)s->ss_parts_cap * rows));
     TRY_ALLOC(dev_alloc(&s->logits, (size_t)s->Q * s->L * V));

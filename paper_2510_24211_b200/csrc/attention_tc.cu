@@ -36,8 +36,9 @@ constexpr unsigned ATT_SPIN_LIMIT = 1u << 22;
 
 struct AttnParams {
     CUtensorMap kv_map;                // the whole pool as a 2-D bf16 matrix [rows][head_dim]
-    const __nv_bfloat16 *qkv;          // [rows][(H + 2 Hkv) dh], Q and K not yet rotated
-    __nv_bfloat16 *out;                // [rows][H dh]
+    const float *qkv;                  // [rows][(H + 2 Hkv) dh] fp32 projections, Q and K not yet rotated
+    __nv_bfloat16 *out;                // [rows][H dh], hi plane; the lo plane (bf16 of the remainder) out_plane elements on
+    long long out_plane;
     __nv_bfloat16 *pool;               // KV pool base (window rows are stored with plain stores)
     const int *page_table;             // [Q][pages_per_seq]
     const int *n_known;                // [B]
@@ -138,29 +139,40 @@ __device__ __forceinline__ uint32_t sw_off(int rows, int row, int col)
     return (uint32_t)(h * rows * 128 + row * 128 + (((c ^ (row & 7)) << 4)) + e * 2);
 }
 
-// RoPE on 8 consecutive pairs (x[j], y[j]) = (dims j0.., dims j0 + dh/2 ..): 16-byte loads of the
-// two halves and of the (cos, sin) table; results scaled and rounded to bf16.
-__device__ __forceinline__ void rotate8(const __nv_bfloat16 *xlo, const __nv_bfloat16 *xhi, const float2 *cs,
+// RoPE on 8 consecutive pairs (x[j], y[j]) = (dims j0.., dims j0 + dh/2 ..) of an fp32 projection row:
+// 16-byte loads of the two halves and of the (cos, sin) table; rotated in fp32, scaled, rounded to bf16 once.
+__device__ __forceinline__ void rotate8(const float *xlo, const float *xhi, const float2 *cs,
                                         float scale, uint4 &out_lo, uint4 &out_hi)
 {
-    const uint4 a = *(const uint4 *)xlo, b = *(const uint4 *)xhi;
+    const float4 a0 = *(const float4 *)xlo, a1 = *(const float4 *)(xlo + 4);
+    const float4 b0 = *(const float4 *)xhi, b1 = *(const float4 *)(xhi + 4);
     const float4 t0 = *(const float4 *)(cs), t1 = *(const float4 *)(cs + 2), t2 = *(const float4 *)(cs + 4),
                  t3 = *(const float4 *)(cs + 6);
     const float c[8] = {t0.x, t0.z, t1.x, t1.z, t2.x, t2.z, t3.x, t3.z};
     const float sn[8] = {t0.y, t0.w, t1.y, t1.w, t2.y, t2.w, t3.y, t3.w};
-    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+    const float x[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+    const float y[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
     uint32_t lo[4], hi[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-        const __nv_bfloat162 av = *reinterpret_cast<const __nv_bfloat162 *>(&aw[k]);
-        const __nv_bfloat162 bv = *reinterpret_cast<const __nv_bfloat162 *>(&bw[k]);
-        const float x0 = __bfloat162float(av.x), x1 = __bfloat162float(av.y);
-        const float y0 = __bfloat162float(bv.x), y1 = __bfloat162float(bv.y);
-        lo[k] = pack_bf16((x0 * c[2 * k] - y0 * sn[2 * k]) * scale, (x1 * c[2 * k + 1] - y1 * sn[2 * k + 1]) * scale);
-        hi[k] = pack_bf16((y0 * c[2 * k] + x0 * sn[2 * k]) * scale, (y1 * c[2 * k + 1] + x1 * sn[2 * k + 1]) * scale);
+        lo[k] = pack_bf16((x[2 * k] * c[2 * k] - y[2 * k] * sn[2 * k]) * scale,
+                          (x[2 * k + 1] * c[2 * k + 1] - y[2 * k + 1] * sn[2 * k + 1]) * scale);
+        hi[k] = pack_bf16((y[2 * k] * c[2 * k] + x[2 * k] * sn[2 * k]) * scale,
+                          (y[2 * k + 1] * c[2 * k + 1] + x[2 * k + 1] * sn[2 * k + 1]) * scale);
     }
     out_lo = make_uint4(lo[0], lo[1], lo[2], lo[3]);
     out_hi = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+}
+// 8 consecutive fp32 values as bf16
+__device__ __forceinline__ uint4 round8(const float *x)
+{
+    const float4 a = *(const float4 *)x, b = *(const float4 *)(x + 4);
+    return make_uint4(pack_bf16(a.x, a.y), pack_bf16(a.z, a.w), pack_bf16(b.x, b.y), pack_bf16(b.z, b.w));
+}
+// the part of (lo, hi) that bf16 drops, as bf16: the second plane of a two-plane activation
+__device__ __forceinline__ uint32_t pack_bf16_rest(float lo, float hi)
+{
+    return pack_bf16(lo - __bfloat162float(__float2bfloat16_rn(lo)), hi - __bfloat162float(__float2bfloat16_rn(hi)));
 }
 
 template <int DH>
@@ -366,7 +378,7 @@ __global__ void __launch_bounds__(256) attention_tc_kernel(const __grid_constant
         if (rr < rows) {
             const int i = rr % Mq, g = rr / Mq;
             const int pos = min(max(base + i, 0), p.max_seq - 1);
-            const __nv_bfloat16 *src = p.qkv + ((size_t)q * Mq + i) * qstride + (size_t)(kvh * p.n_rep + g) * DH;
+            const float *src = p.qkv + ((size_t)q * Mq + i) * qstride + (size_t)(kvh * p.n_rep + g) * DH;
             rotate8(src + j0, src + j0 + half, p.rope + (size_t)pos * half + j0, p.qscale, lo, hi);
         }
         *(uint4 *)(q_s + sw_off(qrows_pad, rr, j0)) = lo;
@@ -435,10 +447,10 @@ __global__ void __launch_bounds__(256) attention_tc_kernel(const __grid_constant
                 uint4 klo = make_uint4(0u, 0u, 0u, 0u), khi = klo, vlo = klo, vhi = klo;
                 const int pos = base + i;
                 if (i < Mq && pos >= 0 && pos < p.max_seq) {
-                    const __nv_bfloat16 *src = p.qkv + ((size_t)q * Mq + i) * qstride + (size_t)(p.H + kvh) * DH;
-                    const __nv_bfloat16 *vs = src + (size_t)p.Hkv * DH;
-                    vlo = *(const uint4 *)(vs + j0);
-                    vhi = *(const uint4 *)(vs + j0 + half);
+                    const float *src = p.qkv + ((size_t)q * Mq + i) * qstride + (size_t)(p.H + kvh) * DH;
+                    const float *vs = src + (size_t)p.Hkv * DH;
+                    vlo = round8(vs + j0);
+                    vhi = round8(vs + j0 + half);
                     rotate8(src + j0, src + j0 + half, p.rope + (size_t)pos * half + j0, 1.0f, klo, khi);
                     const int page = pt[pos >> p.page_shift];
                     const long long r = ((long long)page * p.Hkv + kvh) * p.page_tokens + (pos & (p.page_tokens - 1));
@@ -510,7 +522,9 @@ __global__ void __launch_bounds__(256) attention_tc_kernel(const __grid_constant
 #pragma unroll
                 for (int j = 0; j < DH / 8; ++j) {
                     const int col = j * 8 + 2 * (lane & 3);
-                    *(__nv_bfloat162 *)(dst + col) = __floats2bfloat162_rn(w.o[j][2 * h] * inv, w.o[j][2 * h + 1] * inv);
+                    const float o0 = w.o[j][2 * h] * inv, o1 = w.o[j][2 * h + 1] * inv;
+                    *(__nv_bfloat162 *)(dst + col) = __floats2bfloat162_rn(o0, o1);
+                    *(uint32_t *)(dst + p.out_plane + col) = pack_bf16_rest(o0, o1);
                 }
             }
         }
@@ -578,6 +592,9 @@ __global__ void __launch_bounds__(256) attention_tc_kernel(const __grid_constant
             packed.x = pack_bf16(acc.x, acc.y);
             packed.y = pack_bf16(acc.z, acc.w);
             *(uint2 *)dst = packed;
+            packed.x = pack_bf16_rest(acc.x, acc.y);
+            packed.y = pack_bf16_rest(acc.z, acc.w);
+            *(uint2 *)(dst + p.out_plane) = packed;
         }
     }
     __syncwarp();
@@ -658,8 +675,9 @@ int attention_tc(scd_session *s, int layer, int Mq, int pos_override, cudaStream
     AttnParams p;
     std::memset(&p, 0, sizeof(p));
     p.kv_map = plan->kv_map;
-    p.qkv = (const __nv_bfloat16 *)s->qkv;
+    p.qkv = (const float *)s->qkv;
     p.out = (__nv_bfloat16 *)s->att;
+    p.out_plane = (long long)s->rows_cap * c.n_heads * c.head_dim;
     p.pool = (__nv_bfloat16 *)s->kv_pool;
     p.page_table = s->page_table;
     p.n_known = s->n_known;

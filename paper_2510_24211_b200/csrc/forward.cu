@@ -42,9 +42,10 @@ __device__ __forceinline__ int base_position(const SeqState &s, int q)
 // With `gain` (bf16 sessions) the kernel also prepares the first RMSNorm for the GEMM that follows:
 // xg = bf16(h * gain) and the row's sum of squares (one "partial").
 constexpr int EMBED_THREADS = 512;      // a row of the table is one latency-bound read: many loads in flight
+// `lo_plane` > 0: xg is kept as two planes, xg[lo_plane + .] = T(x - T(x)).
 template <class T>
 __global__ void __launch_bounds__(EMBED_THREADS) embed_kernel(SeqState s, const T *__restrict__ emb, float *__restrict__ h, int d,
-                             const T *__restrict__ gain, T *__restrict__ xg, float *__restrict__ ss_out)
+                             const T *__restrict__ gain, T *__restrict__ xg, float *__restrict__ ss_out, long long lo_plane)
 {
     __shared__ float red[EMBED_THREADS / 32];
     pdl_trigger();
@@ -69,7 +70,13 @@ __global__ void __launch_bounds__(EMBED_THREADS) embed_kernel(SeqState s, const 
     for (int j = threadIdx.x; j < d; j += blockDim.x) {
         const float v = to_f<T>(src[j]);
         dst[j] = v;
-        if (gain) { xg[(size_t)r * d + j] = from_f<T>(v * to_f<T>(gain[j])); ss += v * v; }
+        if (gain) {
+            const float x = v * to_f<T>(gain[j]);
+            const T hi = from_f<T>(x);
+            xg[(size_t)r * d + j] = hi;
+            if (lo_plane > 0) xg[lo_plane + (size_t)r * d + j] = from_f<T>(x - to_f<T>(hi));
+            ss += v * v;
+        }
     }
     if (gain) {
         ss = warp_sum_f(ss);
@@ -169,8 +176,9 @@ __device__ __forceinline__ size_t kv_offset(const KvLayout &kv, int q, int pos, 
     return (((size_t)page * kv.n_kv_heads + kvh) * kv.page_tokens + (pos & (kv.page_tokens - 1))) * kv.head_dim;
 }
 
-template <class T>
-__global__ void rope_kv_kernel(SeqState s, T *__restrict__ qkv, KvLayout kv, const float2 *__restrict__ rope,
+// TQ: type of the projections in qkv (fp32 when they come from the tensor-core GEMM, else T).
+template <class T, class TQ>
+__global__ void rope_kv_kernel(SeqState s, TQ *__restrict__ qkv, KvLayout kv, const float2 *__restrict__ rope,
                                int n_heads)
 {
     pdl_trigger();
@@ -180,28 +188,28 @@ __global__ void rope_kv_kernel(SeqState s, T *__restrict__ qkv, KvLayout kv, con
     const bool in_range = pos >= 0 && pos < kv.max_seq;
     const int pc = min(max(pos, 0), kv.max_seq - 1);
     const float2 *cs = rope + (size_t)pc * half;
-    T *row = qkv + (size_t)r * (n_heads + 2 * Hkv) * dh;
+    TQ *row = qkv + (size_t)r * (n_heads + 2 * Hkv) * dh;
     // Q heads: rotate in place
     for (int e = threadIdx.x; e < n_heads * half; e += blockDim.x) {
         const int hh = e / half, j = e % half;
-        T *v = row + (size_t)hh * dh;
-        const float a = to_f<T>(v[j]), b = to_f<T>(v[j + half]);
+        TQ *v = row + (size_t)hh * dh;
+        const float a = to_f<TQ>(v[j]), b = to_f<TQ>(v[j + half]);
         const float2 t = cs[j];
-        v[j] = from_f<T>(a * t.x - b * t.y);
-        v[j + half] = from_f<T>(b * t.x + a * t.y);
+        v[j] = from_f<TQ>(a * t.x - b * t.y);
+        v[j + half] = from_f<TQ>(b * t.x + a * t.y);
     }
     if (!in_range) return;
     // K heads: rotate into the cache; V heads: copy into the cache
-    const T *krow = row + (size_t)n_heads * dh, *vrow = krow + (size_t)Hkv * dh;
+    const TQ *krow = row + (size_t)n_heads * dh, *vrow = krow + (size_t)Hkv * dh;
     for (int e = threadIdx.x; e < Hkv * half; e += blockDim.x) {
         const int hh = e / half, j = e % half;
-        const float a = to_f<T>(krow[hh * dh + j]), b = to_f<T>(krow[hh * dh + j + half]);
+        const float a = to_f<TQ>(krow[hh * dh + j]), b = to_f<TQ>(krow[hh * dh + j + half]);
         const float2 t = cs[j];
         const size_t o = kv_offset<T>(kv, q, pos, hh);
         ((T *)kv.k_pool)[o + j] = from_f<T>(a * t.x - b * t.y);
         ((T *)kv.k_pool)[o + j + half] = from_f<T>(b * t.x + a * t.y);
-        ((T *)kv.v_pool)[o + j] = vrow[hh * dh + j];
-        ((T *)kv.v_pool)[o + j + half] = vrow[hh * dh + j + half];
+        ((T *)kv.v_pool)[o + j] = from_f<T>(to_f<TQ>(vrow[hh * dh + j]));
+        ((T *)kv.v_pool)[o + j + half] = from_f<T>(to_f<TQ>(vrow[hh * dh + j + half]));
     }
 }
 
@@ -212,9 +220,10 @@ __global__ void rope_kv_kernel(SeqState s, T *__restrict__ qkv, KvLayout kv, con
 constexpr int AQ = 16;           // queries per CTA (4 warps x 4 queries)
 constexpr int AKT = 32;          // keys per tile
 
-template <class T>
-__global__ void __launch_bounds__(128) attention_kernel(SeqState s, const T *__restrict__ qkv, KvLayout kv,
-                                                        T *__restrict__ out, int n_heads, float scale)
+// `lo_plane` > 0: the output is kept as two planes (out[lo_plane + .] = T(o - T(o))).
+template <class T, class TQ>
+__global__ void __launch_bounds__(128) attention_kernel(SeqState s, const TQ *__restrict__ qkv, KvLayout kv,
+                                                        T *__restrict__ out, int n_heads, float scale, long long lo_plane)
 {
     extern __shared__ float smem[];
     pdl_trigger();
@@ -233,7 +242,7 @@ __global__ void __launch_bounds__(128) attention_kernel(SeqState s, const T *__r
 
     for (int e = tid; e < nq * dh; e += blockDim.x) {
         const int qi = e / dh, j = e % dh;
-        qs[qi * dh + j] = to_f<T>(qkv[((size_t)q * s.Mq + i0 + qi) * qstride + (size_t)hh * dh + j]) * scale;
+        qs[qi * dh + j] = to_f<TQ>(qkv[((size_t)q * s.Mq + i0 + qi) * qstride + (size_t)hh * dh + j]) * scale;
     }
     float m[4], l[4], acc[4][4];
 #pragma unroll
@@ -296,7 +305,12 @@ __global__ void __launch_bounds__(128) attention_kernel(SeqState s, const T *__r
         T *o = out + ((size_t)q * s.Mq + i0 + qi) * (size_t)n_heads * dh + (size_t)hh * dh;
 #pragma unroll
         for (int c = 0; c < 4; ++c)
-            if (c < dpl) o[lane + 32 * c] = from_f<T>(acc[a][c] * inv);
+            if (c < dpl) {
+                const float x = acc[a][c] * inv;
+                const T hi = from_f<T>(x);
+                o[lane + 32 * c] = hi;
+                if (lo_plane > 0) o[lo_plane + lane + 32 * c] = from_f<T>(x - to_f<T>(hi));
+            }
     }
 }
 
@@ -347,7 +361,8 @@ int forward_impl(scd_session *s, const ForwardArgs &a, cudaStream_t st)
     // of squares the producer of xn left per row
     int parts = 1;
     embed_kernel<T><<<rows, EMBED_THREADS, 0, st>>>(ss, (const T *)m->tok_emb, s->h, d,
-                                          tc ? (const T *)m->attn_norm[0] : nullptr, xn, s->ss);
+                                          tc ? (const T *)m->attn_norm[0] : nullptr, xn, s->ss,
+                                          tc ? (long long)s->rows_cap * d : 0ll);
     count_launches(1);
 
     KvLayout kv;
@@ -380,11 +395,20 @@ int forward_impl(scd_session *s, const ForwardArgs &a, cudaStream_t st)
             if (rc != SCD_OK) return rc;
         } else {
             MARK(PROF_ROPE_KV);
-            rope_kv_kernel<T><<<rows, 128, 0, st>>>(ss, qkv, kv, m->rope_table, H);
-            count_launches(1);
-            MARK(PROF_ATTENTION);
             dim3 agrid((unsigned)(s->Q * H), (unsigned)((a.Mq + AQ - 1) / AQ));
-            attention_kernel<T><<<agrid, 128, att_smem, st>>>(ss, qkv, kv, att, H, scale);
+            if (tc) {
+                // (projections in fp32 from the tensor-core GEMM; the output in two planes for the next one)
+                rope_kv_kernel<T, float><<<rows, 128, 0, st>>>(ss, (float *)s->qkv, kv, m->rope_table, H);
+                count_launches(1);
+                MARK(PROF_ATTENTION);
+                attention_kernel<T, float><<<agrid, 128, att_smem, st>>>(ss, (const float *)s->qkv, kv, att, H, scale,
+                                                                         (long long)s->rows_cap * dq);
+            } else {
+                rope_kv_kernel<T, T><<<rows, 128, 0, st>>>(ss, qkv, kv, m->rope_table, H);
+                count_launches(1);
+                MARK(PROF_ATTENTION);
+                attention_kernel<T, T><<<agrid, 128, att_smem, st>>>(ss, qkv, kv, att, H, scale, 0ll);
+            }
             count_launches(1);
         }
         MARK(PROF_GEMM_O);

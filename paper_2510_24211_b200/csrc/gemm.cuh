@@ -4,17 +4,19 @@
 
 namespace scd {
 
-// In bf16 sessions the RMSNorm is folded into the GEMMs: s->xn holds bf16(h * gain) and s->ss the
+// In bf16 sessions the RMSNorm is folded into the GEMMs: s->xn holds h * gain and s->ss the
 // partial sums of squares of h ([parts][rows_cap]); a GEMM that reads xn scales its output rows by
 // 1 / rms, a residual GEMM refreshes h, xn (with the gain of the NEXT norm) and ss.
-// qkv[rows][(H+2Hkv)*dh] = norm(h) * [Wq; Wk; Wv]^T                          (bf16 out)
+// Every GEMM input of a session (xn, att, act) is kept as two bf16 planes [2][rows_cap][K]: hi = bf16(x),
+// lo = bf16(x - hi); the GEMMs multiply the weights with both.
+// qkv[rows][(H+2Hkv)*dh] = norm(h) * [Wq; Wk; Wv]^T                          (fp32 out)
 int gemm_tc_qkv(scd_session *s, int layer, int rows, int ss_parts, cudaStream_t st);
 // which = 0: h += att * Wo^T;  which = 1: h += act * Wdown^T                   (fp32 residual)
 // then xn = bf16(h * gain_next), ss = per-tile sums of h^2
 // *parts_out = partial sums of squares it left per row (to be passed to the GEMM that reads xn)
 int gemm_tc_residual(scd_session *s, int layer, int which, int rows, const void *gain_next, int *parts_out,
                      cudaStream_t st);
-// act[rows][F] = silu(norm(h) * Wgate^T) * (norm(h) * Wup^T)                    (bf16 out)
+// act[rows][F] = silu(norm(h) * Wgate^T) * (norm(h) * Wup^T)                    (two bf16 planes out)
 int gemm_tc_gate_up(scd_session *s, int layer, int rows, int ss_parts, cudaStream_t st);
 // logits[rows][v] = norm(h) * Wlm[v]^T for lo <= v < hi and, if eol >= 0, for v = eol    (fp32 out)
 int gemm_tc_lm_head(scd_session *s, int rows, float *logits, int lo, int hi, int eol, int ss_parts, cudaStream_t st);

@@ -27,6 +27,12 @@
 // depends on that kernel (the x operand, the residual stream, the norm statistics) is touched
 // only after the wait.
 //
+// Activations in two bf16 planes: a session keeps every GEMM input x as x_hi = bf16(x) and
+// x_lo = bf16(x - x_hi) (16 significant bits together) and the kernel accumulates W x_hi + W x_lo into the
+// same tensor-memory accumulator - twice the tensor-core work, which the weight stream hides, no extra HBM
+// traffic, and the rounding of the activations drops out of the result (at 32 layers of the 7B shape it
+// was the larger part of the distance to an fp32 evaluation). Weights stay single bf16 values.
+//
 // Fused operations
 //   RMSNorm of the x rows: x holds bf16(h * gain) (not yet divided by the RMS); the sums of
 //     squares of h arrive as `ss_parts` partial sums per row, and the accumulator column of row m
@@ -70,6 +76,8 @@ struct GemmParams {
     int n_seg;
     int M;                           // live window rows
     int nbox;                        // rows of the x box = UMMA N (multiple of 16)
+    int x_planes;                    // 1: x is one bf16 matrix (2-D map); 2: hi and lo plane [2][rows][K] (3-D map)
+    long long out_plane;             // EPI_SWIGLU / xg_out: elements from the hi plane to the lo plane of the output (0: hi only)
     int k_blocks;                    // K / 64
     int k_splits;                    // = cluster size
     int tile_rows;                   // weight rows per tile (<= 128; SwiGLU: features per tile, <= 64)
@@ -121,6 +129,14 @@ __device__ __forceinline__ void tma_load_2d(const CUtensorMap *map, uint64_t *ba
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
                  " [%0], [%1, {%3, %4}], [%2], %5;"
                  ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y), "l"(policy)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(const CUtensorMap *map, uint64_t *bar, void *dst, int x, int y, int z,
+                                            uint64_t policy)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+                 " [%0], [%1, {%3, %4, %5}], [%2], %6;"
+                 ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "l"(policy)
                  : "memory");
 }
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap *map)
@@ -262,6 +278,16 @@ __device__ __forceinline__ void store_bf16x4(__nv_bfloat16 *dst, float4 v, int n
     if (n_ok > 3) dst[3] = __float2bfloat16_rn(v.w);
 }
 
+// v as two bf16 planes: hi = bf16(v), lo = bf16(v - hi)
+__device__ __forceinline__ void store_bf16x4_split(__nv_bfloat16 *hi, long long plane, float4 v, int n_ok, bool vec)
+{
+    store_bf16x4(hi, v, n_ok, vec);
+    if (plane == 0) return;
+    const float4 r = make_float4(v.x - __bfloat162float(__float2bfloat16_rn(v.x)), v.y - __bfloat162float(__float2bfloat16_rn(v.y)),
+                                 v.z - __bfloat162float(__float2bfloat16_rn(v.z)), v.w - __bfloat162float(__float2bfloat16_rn(v.w)));
+    store_bf16x4(hi + plane, r, n_ok, vec);
+}
+
 // Plain outputs (bf16 | fp32 | residual). Epilogue warp `ew` takes window rows m_lo + ew, + 4, ...;
 // R of them per round, the loads from all peers for all R in flight before the first sum. The sum
 // over the peers runs in peer order 0..C-1 for every element.
@@ -309,8 +335,9 @@ __device__ __forceinline__ void reduce_rows(const GemmParams &p, uint32_t base, 
                 hn.x += v.x; hn.y += v.y; hn.z += v.z; hn.w += v.w;
                 store_f32x4((float *)p.out + o, hn, oc);
                 if (norm_out) {
-                    store_bf16x4(p.xg_out + o, make_float4(hn.x * oc.gain.x, hn.y * oc.gain.y, hn.z * oc.gain.z, hn.w * oc.gain.w),
-                                 oc.n_ok, oc.vec);
+                    store_bf16x4_split(p.xg_out + o, p.out_plane,
+                                       make_float4(hn.x * oc.gain.x, hn.y * oc.gain.y, hn.z * oc.gain.z, hn.w * oc.gain.w),
+                                       oc.n_ok, oc.vec);
                     // columns that do not exist hold h = 0; fixed-shape tree over the tile's 128 columns
                     float sq = (hn.x * hn.x + hn.y * hn.y) + (hn.z * hn.z + hn.w * hn.w);
 #pragma unroll
@@ -363,7 +390,7 @@ __device__ __forceinline__ void reduce_swiglu(const GemmParams &p, uint32_t base
             }
             const float4 y = make_float4(g.x / (1.0f + expf(-g.x)) * u.x, g.y / (1.0f + expf(-g.y)) * u.y,
                                          g.z / (1.0f + expf(-g.z)) * u.z, g.w / (1.0f + expf(-g.w)) * u.w);
-            store_bf16x4((__nv_bfloat16 *)p.out + (size_t)m * p.ldo + col, y, n_ok, vec);
+            store_bf16x4_split((__nv_bfloat16 *)p.out + (size_t)m * p.ldo + col, p.out_plane, y, n_ok, vec);
         }
     }
 }
@@ -394,7 +421,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 3) gemm_ws_kernel(const __grid_c
     const int row0 = p.seg_row0[seg] + (tile - p.seg_tile0[seg]) * p.tile_rows;
 
     uint8_t *stage_base = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    const uint32_t a_bytes = TILE_N * BLOCK_K * 2, b_bytes = (uint32_t)nbox * BLOCK_K * 2;
+    const uint32_t a_bytes = TILE_N * BLOCK_K * 2, b_plane = (uint32_t)nbox * BLOCK_K * 2;
+    const uint32_t b_bytes = b_plane * (uint32_t)p.x_planes;      // hi tile, then lo tile
     const uint32_t stage_bytes = a_bytes + b_bytes;
     // bytes one K block brings: the tile's weight rows (the TMA box is tile_rows high) and the x rows
     const uint32_t load_bytes = (uint32_t)p.tile_rows * 128u * (pair ? 2u : 1u) + b_bytes;
@@ -427,8 +455,14 @@ __global__ void __launch_bounds__(GEMM_THREADS, 3) gemm_ws_kernel(const __grid_c
         }
         tma_prefetch_desc(&p.tmap_x);
     }
+    // Two planes of up to 128 rows: ONE instruction per K step multiplies the weight tile with the hi and
+    // the lo tile together (they lie back to back in the slot: a B operand of 2 nbox rows); accumulator
+    // columns [0, nbox) receive W x_hi, [nbox, 2 nbox) W x_lo, and the epilogue adds the halves. The
+    // weight tile is then read from shared memory once per K step, not twice.
+    const bool fused2 = p.x_planes == 2 && 2 * nbox <= 256;
+    const int acc_cols = fused2 ? 2 * nbox : nbox;
     uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < nbox) tmem_cols <<= 1;
+    while ((int)tmem_cols < acc_cols) tmem_cols <<= 1;
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&tmem_base_s)), "r"(tmem_cols) : "memory");
@@ -450,17 +484,20 @@ __global__ void __launch_bounds__(GEMM_THREADS, 3) gemm_ws_kernel(const __grid_c
     if (warp == 0 && lane == 0) {
         // ---------------- TMA producer ----------------
         pdl_wait();                                    // x is written by the kernel in front
-        for (int i = 0; i < pre; ++i)
-            tma_load_2d(&p.tmap_x, &full_bar[i], stage_base + (size_t)i * stage_bytes + a_bytes,
-                        (kb0 + i) * BLOCK_K, 0, pol_x);
+        auto load_x = [&](int i, int s) {
+            uint8_t *sb = stage_base + (size_t)s * stage_bytes + a_bytes;
+            // (two planes: one copy of the box [2][nbox][64] - the hi tile, then the lo tile)
+            if (p.x_planes == 2) tma_load_3d(&p.tmap_x, &full_bar[s], sb, (kb0 + i) * BLOCK_K, 0, 0, pol_x);
+            else tma_load_2d(&p.tmap_x, &full_bar[s], sb, (kb0 + i) * BLOCK_K, 0, pol_x);
+        };
+        for (int i = 0; i < pre; ++i) load_x(i, i);
         int issued = pre;
         for (int i = pre; i < nk; ++i) {
             const int s = i % p.stages, round = i / p.stages;
             if (!mbar_wait(&empty_bar[s], (round & 1) ^ 1)) { atomicExch(p.err, 1); abort_flag = 1; break; }
             mbar_expect_tx(&full_bar[s], load_bytes);
             load_w(i, s);
-            tma_load_2d(&p.tmap_x, &full_bar[s], stage_base + (size_t)s * stage_bytes + a_bytes,
-                        (kb0 + i) * BLOCK_K, 0, pol_x);
+            load_x(i, s);
             issued = i + 1;
         }
         if (abort_flag) {
@@ -470,7 +507,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 3) gemm_ws_kernel(const __grid_c
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------- MMA issuer ----------------
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(nbox >> 3) << 17) |
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(acc_cols >> 3) << 17) |
                                ((uint32_t)(TILE_N >> 4) << 24);
         bool ok = true;
         for (int i = 0; i < nk && ok; ++i) {
@@ -484,6 +521,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 3) gemm_ws_kernel(const __grid_c
             for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
                 const uint32_t koff = k * UMMA_K * 2;
                 umma_bf16(tmem_base, umma_desc(sa + koff), umma_desc(sb + koff), idesc, (i > 0 || k > 0) ? 1u : 0u);
+                if (p.x_planes == 2 && !fused2) umma_bf16(tmem_base, umma_desc(sa + koff), umma_desc(sb + b_plane + koff), idesc, 1u);
             }
             umma_commit(&empty_bar[s]);        // frees the slot once these MMAs have read it
         }
@@ -537,12 +575,24 @@ __global__ void __launch_bounds__(GEMM_THREADS, 3) gemm_ws_kernel(const __grid_c
             for (; c + 32 <= nbox; c += 32) {            // 32 accumulator columns per tensor-memory load
                 float v[32];
                 tmem_ld32(taddr + c, v);
+                if (fused2) {
+                    float v2[32];
+                    tmem_ld32(taddr + nbox + c, v2);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] += v2[j];
+                }
 #pragma unroll
                 for (int j = 0; j < 32; ++j) stage_part[(size_t)(c + j) * TILE_N + r] = v[j];
             }
             for (; c < nbox; c += 16) {
                 float v[16];
                 tmem_ld16(taddr + c, v);
+                if (fused2) {
+                    float v2[16];
+                    tmem_ld16(taddr + nbox + c, v2);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] += v2[j];
+                }
 #pragma unroll
                 for (int j = 0; j < 16; ++j) stage_part[(size_t)(c + j) * TILE_N + r] = v[j];
             }
@@ -620,6 +670,23 @@ int make_map(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t K, uint3
     return make_tensor_map_bf16_2d(map, ptr, rows, K, box_rows, BLOCK_K);
 }
 
+// Two-plane activation buffer [2][rows][K] bf16: box = 64 (K) x box_rows x both planes, 128-byte swizzle.
+int make_map_planes(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t K, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    SCD_REQUIRE(fn, SCD_ERR_CUDA, "cuTensorMapEncodeTiled entry point not found");
+    cuuint64_t dims[3] = {K, rows, 2};
+    cuuint64_t strides[2] = {K * 2, rows * K * 2};
+    cuuint32_t box[3] = {BLOCK_K, box_rows, 2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    SCD_REQUIRE(r == CUDA_SUCCESS, SCD_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) rows %llu K %llu box rows %u, two planes",
+                (int)r, (unsigned long long)rows, (unsigned long long)K, box_rows);
+    return SCD_OK;
+}
+
 struct GemmPlan {                    // per model: weight-side tensor maps, built on first use
     std::map<std::tuple<const void *, int, int, int>, CUtensorMap> wmaps;   // (matrix, rows, K, box rows)
     int sm_count;
@@ -629,7 +696,7 @@ struct GemmPlan {                    // per model: weight-side tensor maps, buil
 
 inline int round16(int m) { return std::max(16, (m + 15) & ~15); }
 
-inline size_t stage_bytes_of(int nbox) { return (size_t)TILE_N * BLOCK_K * 2 + (size_t)nbox * BLOCK_K * 2; }
+inline size_t stage_bytes_of(int nbox, int planes) { return (size_t)TILE_N * BLOCK_K * 2 + (size_t)planes * nbox * BLOCK_K * 2; }
 inline size_t staging_bytes_of(int nbox) { return (size_t)nbox * TILE_N * sizeof(float); }
 constexpr size_t SMEM_LIMIT = 227 * 1024 - 8192;   // dynamic shared memory one CTA may ask for
 
@@ -667,9 +734,9 @@ void choose_shape(const Segment *segs, int n_seg, bool pair, int k_blocks, int s
 // Ring slots: about 72 KB per CTA so that three CTAs share an SM - or about 100 KB when the grid has
 // at most two CTAs per SM anyway (measured: the deeper ring then wins a few percent) - and never
 // less than the partial-tile staging.
-int choose_stages(int nbox, int k_blocks_per_cta, bool two_per_sm, int forced = 0)
+int choose_stages(int nbox, int planes, int k_blocks_per_cta, bool two_per_sm, int forced = 0)
 {
-    const int stage_bytes = (int)stage_bytes_of(nbox);
+    const int stage_bytes = (int)stage_bytes_of(nbox, planes);
     int st = std::max(2, ((two_per_sm ? 100 : 73) * 1024) / stage_bytes);
     if (forced > 0) st = forced;
     st = std::min(st, (int)((SMEM_LIMIT - 1024) / stage_bytes));
@@ -680,7 +747,7 @@ int choose_stages(int nbox, int k_blocks_per_cta, bool two_per_sm, int forced = 
 
 int launch(GemmParams &p, int tiles, cudaStream_t st)
 {
-    const size_t ring = std::max((size_t)p.stages * stage_bytes_of(p.nbox), staging_bytes_of(p.nbox));
+    const size_t ring = std::max((size_t)p.stages * stage_bytes_of(p.nbox, p.x_planes), staging_bytes_of(p.nbox));
     p.aux_offset = (int)ring;
     const size_t rows_per_cta = (size_t)(p.M + p.k_splits - 1) / p.k_splits;
     size_t smem = ring + 5 * rows_per_cta * sizeof(float) + 1024;
@@ -719,6 +786,7 @@ struct SessionGemm {                 // activation-side tensor maps of a session
     std::map<std::tuple<const void *, int, int>, CUtensorMap> xmaps;
 };
 
+// (both planes of an activation buffer in one map)
 int x_map(scd_session *s, const void *buf, int K, int nbox, CUtensorMap *out)
 {
     SessionGemm *sg = (SessionGemm *)s->gemm_state;
@@ -726,7 +794,7 @@ int x_map(scd_session *s, const void *buf, int K, int nbox, CUtensorMap *out)
     auto it = sg->xmaps.find(key);
     if (it == sg->xmaps.end()) {
         CUtensorMap m;
-        int rc = make_map(&m, buf, (uint64_t)s->rows_cap, (uint64_t)K, (uint32_t)nbox);
+        int rc = make_map_planes(&m, buf, (uint64_t)s->rows_cap, (uint64_t)K, (uint32_t)nbox);
         if (rc != SCD_OK) return rc;
         it = sg->xmaps.emplace(key, m).first;
     }
@@ -778,8 +846,10 @@ int run_gemm(scd_session *s, int kind, const Segment *segs, int n_seg, int epi, 
     p.n_seg = pair ? 1 : n_seg;
     p.M = rows;
     p.nbox = round16(rows);
-    p.stages = choose_stages(p.nbox, (p.k_blocks + p.k_splits - 1) / p.k_splits, tiles * p.k_splits <= 2 * plan->sm_count,
-                             plan->forced_stages);
+    p.x_planes = 2;
+    p.out_plane = (long long)s->rows_cap * ldo;           // (used by the outputs that are GEMM inputs themselves)
+    p.stages = choose_stages(p.nbox, p.x_planes, (p.k_blocks + p.k_splits - 1) / p.k_splits,
+                             tiles * p.k_splits <= 2 * plan->sm_count, plan->forced_stages);
     p.epi = epi;
     p.out = out;
     p.ldo = ldo;
@@ -832,7 +902,8 @@ int gemm_tc_qkv(scd_session *s, int l, int rows, int ss_parts, cudaStream_t st)
     const int d = c.d_model, dq = c.n_heads * c.head_dim, dkv = c.n_kv_heads * c.head_dim;
     const Segment segs[3] = {{m->wq[l], dq, d, 0, dq, 0}, {m->wk[l], dkv, d, 0, dkv, dq}, {m->wv[l], dkv, d, 0, dkv, dq + dkv}};
     const NormIn nin = {s->ss, ss_parts};
-    return run_gemm(s, GEMM_QKV, segs, 3, EPI_BF16, s->xn, d, rows, s->qkv, dq + 2 * dkv, &nin, nullptr, st);
+    // fp32 out: the attention kernel rotates Q and K in fp32 and rounds each of Q, K, V to bf16 once
+    return run_gemm(s, GEMM_QKV, segs, 3, EPI_F32, s->xn, d, rows, s->qkv, dq + 2 * dkv, &nin, nullptr, st);
 }
 
 int gemm_tc_residual(scd_session *s, int l, int which, int rows, const void *gain_next, int *parts_out,
@@ -961,7 +1032,8 @@ int scd_gemm_bf16_shaped(const void *x, const void *w, float *y, int32_t M, int3
     if (rc != SCD_OK) return rc;
     p.seg_tile0[0] = 0; p.seg_tile0[1] = tiles; p.seg_row0[0] = 0; p.seg_nout[0] = N; p.seg_col0[0] = 0; p.n_seg = 1;
     p.M = M;
-    p.stages = choose_stages(p.nbox, (p.k_blocks + p.k_splits - 1) / p.k_splits, tiles * p.k_splits <= 2 * sms, stages);
+    p.x_planes = 1;                                       // the hook multiplies one bf16 matrix
+    p.stages = choose_stages(p.nbox, 1, (p.k_blocks + p.k_splits - 1) / p.k_splits, tiles * p.k_splits <= 2 * sms, stages);
     p.epi = EPI_F32;
     p.out = y;
     p.ldo = N;
