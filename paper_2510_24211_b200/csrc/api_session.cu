@@ -17,6 +17,8 @@ void count_launches(long long n) { g_launches.fetch_add(n, std::memory_order_rel
 
 namespace {
 
+constexpr int GENERATE_BLOCK = 64;      // iterations scd_generate enqueues between two looks at the counters
+
 inline bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
 inline size_t elem_size(int dtype) { return dtype == SCD_F32 ? 4 : 2; }
 
@@ -71,6 +73,7 @@ void session_verify_params(scd_session *s, VerifyParams &p)
     p.row_y = s->row_y; p.row_y_indep = s->row_y_indep;
     p.done_count = s->done_count;
     p.dev_stats = s->dev_stats;
+    p.finished = s->finished;
 }
 
 int enqueue_step(scd_session *s, cudaStream_t st, StepProfiler *prof = nullptr)
@@ -78,6 +81,7 @@ int enqueue_step(scd_session *s, cudaStream_t st, StepProfiler *prof = nullptr)
     ForwardArgs a;
     a.ids = nullptr; a.Mq = s->L; a.pos_override = -1; a.want_logits = true;
     a.logits = s->logits; a.hidden = nullptr; a.prof = prof;
+    a.skip = s->finished + 1;                            // an iteration enqueued after the last token costs only its launches
     // the sampler reads only the ids it may draw: the allowed range and the end-of-row id
     a.lm_lo = s->cfg.allowed_lo; a.lm_hi = s->cfg.allowed_hi;
     a.lm_eol = s->cfg.row_period > 0 ? s->cfg.eol_id : -1;
@@ -148,7 +152,7 @@ void free_session_memory(scd_session *s)
     void *ptrs[] = {s->kv_pool, s->page_table, s->n_known, s->n_total, s->shift, s->prev_lw, s->drafts,
                     s->n_commit, s->tokens, s->tokens_u, s->row_y, s->row_y_indep, s->ids_buf, s->iter,
                     s->done_count, s->accept_flags, s->xbuf[0], s->xbuf[1], s->stats[0], s->stats[1],
-                    s->dev_stats, s->h, s->ss, s->xn, s->qkv, s->att, s->gu, s->act, s->logits, s->gemm_ws, s->stamps};
+                    s->dev_stats, s->finished, s->h, s->ss, s->xn, s->qkv, s->att, s->gu, s->act, s->logits, s->gemm_ws, s->stamps};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (s->host_pinned) cudaFreeHost(s->host_pinned);
     if (s->gemm_state) gemm_session_release(s);
@@ -287,6 +291,7 @@ int scd_session_create(scd_model_t *m, const scd_decode_config_t *cfg, scd_sessi
     TRY_ALLOC(dev_alloc(&s->stats[0], wrows));
     TRY_ALLOC(dev_alloc(&s->stats[1], wrows));
     TRY_ALLOC(dev_alloc(&s->dev_stats, 1));
+    TRY_ALLOC(dev_alloc(&s->finished, 2));
     TRY_ALLOC(dev_alloc(&s->h, rows * d));
     // bf16 sessions: GEMM inputs (xn, att, act) in two bf16 planes [2][rows][K], projections (qkv) in fp32
     const size_t wide = c.dtype == SCD_BF16 ? 2 : 1;
@@ -354,23 +359,19 @@ int scd_prefill(scd_session_t *s, const int32_t *prompt_ids, int32_t P, int32_t 
         SCD_CUDA_TRY(cudaMemcpy2DAsync(s->tokens_u, (size_t)c.max_seq * sizeof(int),
                                        s->host_pinned + (size_t)s->B * P, (size_t)P * sizeof(int),
                                        (size_t)P * sizeof(int), s->B, cudaMemcpyHostToDevice, st));
-    SCD_CUDA_TRY(cudaStreamSynchronize(st));
-    // chunks of the prompt (all but its last token) through the forward, no logits
+    // chunks of the prompt (all but its last token) through the forward, no logits; the kernels read the
+    // prompt from the token records just copied, so the chunks are enqueued back to back
     for (int p0 = 0; p0 < P - 1; p0 += s->chunk) {
         const int len = std::min(s->chunk, P - 1 - p0);
-        for (int q = 0; q < s->Q; ++q)
-            std::memcpy(s->host_pinned + (size_t)q * len, prompt_ids + (size_t)q * P + p0, (size_t)len * sizeof(int));
-        SCD_CUDA_TRY(cudaMemcpyAsync(s->ids_buf, s->host_pinned, (size_t)s->Q * len * sizeof(int),
-                                     cudaMemcpyHostToDevice, st));
         ForwardArgs a;
-        a.ids = s->ids_buf; a.Mq = len; a.pos_override = p0; a.want_logits = false;
+        a.ids = nullptr; a.Mq = len; a.pos_override = p0; a.want_logits = false; a.skip = nullptr;
         a.logits = nullptr; a.hidden = nullptr; a.prof = nullptr; a.lm_lo = 0; a.lm_hi = 0; a.lm_eol = -1;
         int rc = run_forward(s, a, st);
         if (rc != SCD_OK) return rc;
-        SCD_CUDA_TRY(cudaStreamSynchronize(st));
     }
     set_state_kernel<<<(s->B + 63) / 64, 64, 0, st>>>(s->n_known, s->n_total, s->B, P, P + n_new);
     SCD_CUDA_TRY(cudaMemsetAsync(s->dev_stats, 0, sizeof(VerifyStatsDev), st));
+    SCD_CUDA_TRY(cudaMemsetAsync(s->finished, 0, 2 * sizeof(int), st));
     VerifyParams p;
     session_verify_params(s, p);
     int rc = launch_init_window(p, st);
@@ -414,7 +415,7 @@ int scd_autotune(scd_session_t *s, int32_t *k_splits_out, void *stream)
     drop_step_graph(s);                                  // the captured launches carry the old shapes
     ForwardArgs a;
     a.ids = nullptr; a.Mq = s->L; a.pos_override = -1; a.want_logits = true;
-    a.logits = s->logits; a.hidden = nullptr; a.prof = nullptr;
+    a.logits = s->logits; a.hidden = nullptr; a.prof = nullptr; a.skip = nullptr;
     a.lm_lo = s->cfg.allowed_lo; a.lm_hi = s->cfg.allowed_hi;
     a.lm_eol = s->cfg.row_period > 0 ? s->cfg.eol_id : -1;
     cudaEvent_t e0, e1;
@@ -530,17 +531,19 @@ int scd_generate(scd_session_t *s, int32_t *out_tokens, scd_stats_t *stats, void
     int rc = SCD_OK;
     long long launched = 0;
     for (;;) {
-        // every iteration commits between 1 and L tokens per unfinished sequence, so
-        // ceil(remaining / L) more iterations are always needed: enqueue them without a host
-        // round trip, then look again.
+        // Every iteration commits between 1 and L tokens per unfinished sequence: `remaining` iterations
+        // always suffice and ceil(remaining / L) are always needed. Iterations are enqueued in blocks of
+        // up to GENERATE_BLOCK without a host round trip; the host looks at the counters once per block.
+        // An iteration that runs after the last token costs only its (empty) launches: the verify kernel
+        // raises a device flag when every sequence is complete and the forward kernels return on it.
         SCD_CUDA_TRY(cudaMemcpyAsync(hp, s->n_known, s->B * sizeof(int), cudaMemcpyDeviceToHost, st));
         SCD_CUDA_TRY(cudaStreamSynchronize(st));
         int remaining = 0;
         for (int b = 0; b < s->B; ++b) remaining = std::max(remaining, total - hp[b]);
         if (remaining <= 0) break;
-        const int steps = (remaining + s->L - 1) / s->L;
+        const int steps = std::max((remaining + s->L - 1) / s->L, std::min(remaining, GENERATE_BLOCK));
         launched += steps;
-        if (launched > (long long)s->n_new + 8) {      // each iteration commits >= 1 token
+        if (launched > (long long)s->n_new + 8 + GENERATE_BLOCK) {      // each live iteration commits >= 1 token
             set_last_error("scd_generate: no progress after %lld iterations", launched);
             rc = SCD_ERR_TIMEOUT;
             break;
@@ -579,7 +582,7 @@ int scd_forward_window(scd_session_t *s, const int32_t *ids, int32_t M, float *l
     cudaStream_t st = (cudaStream_t)stream;
     ForwardArgs a;
     a.ids = ids; a.Mq = M; a.pos_override = -1; a.want_logits = true; a.logits = logits; a.hidden = hidden;
-    a.prof = nullptr; a.lm_lo = 0; a.lm_hi = 0; a.lm_eol = -1;
+    a.prof = nullptr; a.skip = nullptr; a.lm_lo = 0; a.lm_hi = 0; a.lm_eol = -1;
     int rc = run_forward(s, a, st);
     if (rc != SCD_OK) return rc;
     if (commit) {

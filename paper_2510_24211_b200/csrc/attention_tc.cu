@@ -44,6 +44,7 @@ struct AttnParams {
     const int *n_known;                // [B]
     const float2 *rope;                // [max_seq][dh/2] (cos, sin)
     int *err;
+    const int *skip;                   // optional device flag: set = nothing to do, return at once
     long long row0_k, row0_v;          // pool row of (this layer, K | V, page 0, head 0, token 0)
     int B, Mq, H, Hkv, n_rep, pages_per_seq, page_tokens, page_shift, max_seq, pos_override;
     int C, stages, n_mtiles;
@@ -304,6 +305,7 @@ __global__ void __launch_bounds__(256) attention_tc_kernel(const __grid_constant
     __shared__ int abort_flag;
 
     pdl_trigger();                     // the GEMM behind may take the SM slots this grid leaves free
+    if (p.skip && *p.skip) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (p.stamp && tid == 0 && blockIdx.x < STAMP_CTAS) p.stamp[blockIdx.x] = global_timer_ns();
     const int C = p.C, rank = blockIdx.x % C, unit = blockIdx.x / C;
@@ -683,6 +685,7 @@ int attention_tc(scd_session *s, int layer, int Mq, int pos_override, cudaStream
     p.n_known = s->n_known;
     p.rope = s->model->rope_table;
     p.err = (int *)s->gemm_ws;
+    p.skip = s->skip_now;
     p.stamp = take_stamp_slot();
     const long long rows_per_kind = (long long)s->Q * s->pages_per_seq * c.n_kv_heads * c.kv_page_tokens;
     p.row0_k = (long long)layer * 2 * rows_per_kind;

@@ -29,6 +29,7 @@ struct SeqState {             // where window inputs and positions come from
     const int *tokens_u;      // [B][prompt_cap] unconditional prompt
     const int *drafts;        // [B][L]
     int token_stride, prompt_cap, prompt_len, L, B, Mq, pos_override, vocab_in;
+    const int *skip;          // all sequences finished: nothing to do
 };
 
 __device__ __forceinline__ int base_position(const SeqState &s, int q)
@@ -49,10 +50,15 @@ __global__ void __launch_bounds__(EMBED_THREADS) embed_kernel(SeqState s, const 
 {
     __shared__ float red[EMBED_THREADS / 32];
     pdl_trigger();
+    if (s.skip && *s.skip) return;
     const int r = blockIdx.x, q = r / s.Mq, i = r % s.Mq;
     int id;
     if (s.ids) {
         id = s.ids[r];
+    } else if (s.pos_override >= 0) {
+        // prefill: the prompt as recorded on the device (the unconditional stream has its own prompt)
+        const int b = q % s.B, stream = q / s.B, pos = s.pos_override + i;
+        id = stream == 1 ? s.tokens_u[(size_t)b * s.prompt_cap + pos] : s.tokens[(size_t)b * s.token_stride + pos];
     } else {
         const int b = q % s.B, stream = q / s.B;
         if (i == 0) {
@@ -351,7 +357,7 @@ int forward_impl(scd_session *s, const ForwardArgs &a, cudaStream_t st)
     ss.ids = a.ids; ss.n_known = s->n_known; ss.tokens = s->tokens; ss.tokens_u = s->tokens_u;
     ss.drafts = s->drafts; ss.token_stride = c.max_seq; ss.prompt_cap = c.max_seq;
     ss.prompt_len = s->prompt_len; ss.L = s->L; ss.B = s->B; ss.Mq = a.Mq;
-    ss.pos_override = a.pos_override; ss.vocab_in = c.vocab_in;
+    ss.pos_override = a.pos_override; ss.vocab_in = c.vocab_in; ss.skip = a.skip;
 
     T *xn = (T *)s->xn, *qkv = (T *)s->qkv, *att = (T *)s->att, *gu = (T *)s->gu, *act = (T *)s->act;
     StepProfiler *prof = a.prof;
@@ -545,6 +551,7 @@ StepProfiler::~StepProfiler()
 
 int run_forward(scd_session *s, const ForwardArgs &a, cudaStream_t st)
 {
+    s->skip_now = a.skip;
     if (s->model->cfg.dtype == SCD_F32) return forward_impl<float>(s, a, st);
     return forward_impl<__nv_bfloat16>(s, a, st);
 }

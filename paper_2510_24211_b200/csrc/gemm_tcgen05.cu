@@ -95,6 +95,7 @@ struct GemmParams {
     __nv_bfloat16 *xg_out;           // [M][ldo] bf16(h * gain_next)
     float *ss_out;                   // [tiles][ss_stride] this tile's sum of h^2 per row
     int *err;                        // device error word
+    const int *skip;                 // optional device flag: set = nothing to do, return at once
     unsigned long long *stamp;       // optional [2][STAMP_CTAS]: %globaltimer at CTA entry and exit
 };
 
@@ -404,6 +405,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 3) gemm_ws_kernel(const __grid_c
     __shared__ int healthy_s[4];               // per epilogue warp: accumulator complete, no error raised
 
     pdl_trigger();                     // the next kernel may take the SM slots this grid leaves free
+    if (p.skip && *p.skip) return;     // (the flag is older than this iteration: the same answer in every CTA)
     if (p.stamp && threadIdx.x == 0 && blockIdx.x < STAMP_CTAS) p.stamp[blockIdx.x] = global_timer_ns();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int C = p.k_splits;
@@ -865,6 +867,7 @@ int run_gemm(scd_session *s, int kind, const Segment *segs, int n_seg, int epi, 
     int rc = x_map(s, x, K, p.nbox, &p.tmap_x);
     if (rc != SCD_OK) return rc;
     p.err = (int *)s->gemm_ws;
+    p.skip = s->skip_now;
     p.stamp = take_stamp_slot();
     g_last_tiles = tiles;
     return launch(p, tiles, st);

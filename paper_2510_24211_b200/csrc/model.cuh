@@ -38,6 +38,8 @@ struct scd_session {
     float *xbuf[2];
     scd::RowStats *stats[2];
     scd::VerifyStatsDev *dev_stats;
+    int *finished;            // device: [0] finished sequences, [1] all finished (see VerifyParams::finished)
+    const int *skip_now;      // what the forward being enqueued hands its kernels as skip flag (NULL or finished + 1)
 
     // activations (device)
     float *h;                 // residual stream [rows][d]
@@ -92,7 +94,9 @@ struct StepProfiler {
 unsigned long long *take_stamp_slot();
 
 struct ForwardArgs {
-    const int *ids;           // explicit input ids [Q][Mq] (device) or NULL: window inputs from state
+    const int *ids;           // explicit input ids [Q][Mq] (device) or NULL: window inputs from state, or - with
+                              // pos_override >= 0 - the recorded tokens at positions pos_override .. + Mq - 1 (prefill)
+    const int *skip;          // device flag: the kernels return at once when it is set (NULL: never)
     int Mq;                   // rows per stream-sequence
     int pos_override;         // >= 0: position of row 0 for every stream-sequence; < 0: n_known - 1
     bool want_logits;

@@ -741,9 +741,11 @@ __global__ void __launch_bounds__(VT, 1) verify_kernel(const VerifyParams p, int
             p.iter[b] = w.t + 1u;
             p.shift[b] = a;
             p.prev_lw[b] = w.Lw;
+            // this iteration completed the sequence (it was live: Lw > 0): the last of the batch raises the flag
+            if (p.finished && (int)w.pos0 + a >= p.n_total[b] && atomicAdd(&p.finished[0], 1) == p.B - 1) p.finished[1] = 1;
         }
         if (p.dev_stats) {
-            if (b == 0) atomicAdd(&p.dev_stats->forwards, 1ull);
+            atomicMax(&p.dev_stats->forwards, (unsigned long long)w.t + 1ull);   // iterations in which a sequence was live
             atomicAdd(&p.dev_stats->committed, (unsigned long long)a);
             atomicAdd(&p.dev_stats->accept_hist[a], 1ull);
         }

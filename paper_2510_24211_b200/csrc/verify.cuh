@@ -63,6 +63,8 @@ struct VerifyParams {
     int *row_y_indep;             // [2][B][L] scratch: redraft beyond the prefix (SJD, alpha, Gumbel); fresh rows (Gumbel)
     unsigned int *done_count;     // [B] scratch, zero on entry, zero again on exit
     VerifyStatsDev *dev_stats;    // session counters (or NULL)
+    int *finished;                // session: [0] sequences that reached their final length, [1] = 1 once all B have
+                                  // (the forward kernels of an iteration enqueued after that return at once)   (or NULL)
 };
 
 // ---- device helpers shared by the two verify kernels -----------------------------------------------
