@@ -11,7 +11,10 @@
 //     before griddepcontrol.wait, because the cache of earlier iterations does not depend on
 //     the QKV projection that runs in front of this kernel.
 //   - one warp per 16 query rows: S = Q K^T and O += P V on mma.sync m16n8k16 (bf16 in, fp32
-//     accumulate), online softmax in fp32 with base-2 exponentials.
+//     accumulate), online softmax in fp32 with base-2 exponentials. The rotated, scaled queries are
+//     kept as two bf16 planes (value and remainder) and S = Q_hi K^T + Q_lo K^T: the queries are the
+//     one operand of the scores that is not bound to the cache's bf16, and their rounding was a
+//     measurable part of the distance to an fp32 evaluation at full depth.
 //   - each CTA leaves (max, sum, unnormalised O) of its key range in shared memory; after a
 //     cluster barrier CTA c merges the query rows [c R / C, (c+1) R / C) over all peers through
 //     distributed shared memory in peer order, normalises and stores bf16.
@@ -142,8 +145,11 @@ __device__ __forceinline__ uint32_t sw_off(int rows, int row, int col)
 
 // RoPE on 8 consecutive pairs (x[j], y[j]) = (dims j0.., dims j0 + dh/2 ..) of an fp32 projection row:
 // 16-byte loads of the two halves and of the (cos, sin) table; rotated in fp32, scaled, rounded to bf16 once.
+__device__ __forceinline__ uint32_t pack_bf16_rest(float lo, float hi);
+// (rest_lo / rest_hi, when given, receive what the rounding dropped, as bf16: the second plane)
 __device__ __forceinline__ void rotate8(const float *xlo, const float *xhi, const float2 *cs,
-                                        float scale, uint4 &out_lo, uint4 &out_hi)
+                                        float scale, uint4 &out_lo, uint4 &out_hi, uint4 *rest_lo = nullptr,
+                                        uint4 *rest_hi = nullptr)
 {
     const float4 a0 = *(const float4 *)xlo, a1 = *(const float4 *)(xlo + 4);
     const float4 b0 = *(const float4 *)xhi, b1 = *(const float4 *)(xhi + 4);
@@ -153,16 +159,21 @@ __device__ __forceinline__ void rotate8(const float *xlo, const float *xhi, cons
     const float sn[8] = {t0.y, t0.w, t1.y, t1.w, t2.y, t2.w, t3.y, t3.w};
     const float x[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
     const float y[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-    uint32_t lo[4], hi[4];
+    uint32_t lo[4], hi[4], rlo[4], rhi[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-        lo[k] = pack_bf16((x[2 * k] * c[2 * k] - y[2 * k] * sn[2 * k]) * scale,
-                          (x[2 * k + 1] * c[2 * k + 1] - y[2 * k + 1] * sn[2 * k + 1]) * scale);
-        hi[k] = pack_bf16((y[2 * k] * c[2 * k] + x[2 * k] * sn[2 * k]) * scale,
-                          (y[2 * k + 1] * c[2 * k + 1] + x[2 * k + 1] * sn[2 * k + 1]) * scale);
+        const float l0 = (x[2 * k] * c[2 * k] - y[2 * k] * sn[2 * k]) * scale;
+        const float l1 = (x[2 * k + 1] * c[2 * k + 1] - y[2 * k + 1] * sn[2 * k + 1]) * scale;
+        const float h0 = (y[2 * k] * c[2 * k] + x[2 * k] * sn[2 * k]) * scale;
+        const float h1 = (y[2 * k + 1] * c[2 * k + 1] + x[2 * k + 1] * sn[2 * k + 1]) * scale;
+        lo[k] = pack_bf16(l0, l1);
+        hi[k] = pack_bf16(h0, h1);
+        rlo[k] = pack_bf16_rest(l0, l1);
+        rhi[k] = pack_bf16_rest(h0, h1);
     }
     out_lo = make_uint4(lo[0], lo[1], lo[2], lo[3]);
     out_hi = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    if (rest_lo) { *rest_lo = make_uint4(rlo[0], rlo[1], rlo[2], rlo[3]); *rest_hi = make_uint4(rhi[0], rhi[1], rhi[2], rhi[3]); }
 }
 // 8 consecutive fp32 values as bf16
 __device__ __forceinline__ uint4 round8(const float *x)
@@ -181,6 +192,8 @@ struct WarpState {
     uint32_t qf[DH / 16][4];     // Q fragments of this warp's 16 rows
     float o[DH / 8][4];          // unnormalised output
     float m[2], l[2];            // running max / sum of rows g and g + 8
+    uint32_t qlo_base;           // shared-memory address of the queries' remainder plane
+    int q_rows, q_row;           // its row count (padded) and the row this lane addresses in ldmatrix
 };
 
 // One tile of TK keys: S = Q K^T, masking, online softmax, O += P V.
@@ -195,17 +208,21 @@ __device__ __forceinline__ void process_keys(WarpState<DH> &w, uint32_t kbase, u
     float s[KEYS / 8][4];
 #pragma unroll
     for (int n = 0; n < KEYS / 8; ++n) { s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f; }
-    // ---- S = Q K^T ----
+    // ---- S = Q_hi K^T + Q_lo K^T (the remainder fragments come from shared memory, one per K step) ----
 #pragma unroll
-    for (int n2 = 0; n2 < KEYS / 16; ++n2) {
-        const int key = n2 * 16 + ((lane >> 4) << 3) + (lane & 7);
+    for (int ks = 0; ks < DH / 16; ++ks) {
+        uint32_t ql[4];
+        ldsm_x4(w.qlo_base + sw_off(w.q_rows, w.q_row, ks * 16 + ((lane >> 4) << 3)), ql[0], ql[1], ql[2], ql[3]);
 #pragma unroll
-        for (int ks = 0; ks < DH / 16; ++ks) {
+        for (int n2 = 0; n2 < KEYS / 16; ++n2) {
+            const int key = n2 * 16 + ((lane >> 4) << 3) + (lane & 7);
             const int col = ks * 16 + (((lane >> 3) & 1) << 3);
             uint32_t b0, b1, b2, b3;
             ldsm_x4(kbase + sw_off(TK, key, col), b0, b1, b2, b3);
             mma_bf16(s[2 * n2], w.qf[ks], b0, b1);
             mma_bf16(s[2 * n2 + 1], w.qf[ks], b2, b3);
+            mma_bf16(s[2 * n2], ql, b0, b1);
+            mma_bf16(s[2 * n2 + 1], ql, b2, b3);
         }
     }
     // ---- mask ----
@@ -320,8 +337,10 @@ __global__ void __launch_bounds__(256) attention_tc_kernel(const __grid_constant
         if (tid == 0) atomicExch(p.err, 6);
         return;
     }
-    uint8_t *q_s = smem_raw;                                      // [DH/64][qrows_pad][128 B]
-    uint8_t *stages = q_s + (((size_t)qrows_pad * DH * 2 + 1023) & ~(size_t)1023);
+    uint8_t *q_s = smem_raw;                                      // [DH/64][qrows_pad][128 B]: the queries as bf16 ...
+    const size_t q_plane = ((size_t)qrows_pad * DH * 2 + 1023) & ~(size_t)1023;
+    uint8_t *q_lo_s = q_s + q_plane;                              // ... and what bf16 dropped, same layout
+    uint8_t *stages = q_lo_s + q_plane;
 
     if (tid == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], (unsigned)(p.n_mtiles * KS)); }
@@ -376,19 +395,24 @@ __global__ void __launch_bounds__(256) attention_tc_kernel(const __grid_constant
 #pragma unroll 4
     for (int e = tid; e < qrows_pad * CH; e += blockDim.x) {
         const int rr = e / CH, j0 = (e % CH) * 8;
-        uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo;
+        uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo, rlo = lo, rhi = lo;
         if (rr < rows) {
             const int i = rr % Mq, g = rr / Mq;
             const int pos = min(max(base + i, 0), p.max_seq - 1);
             const float *src = p.qkv + ((size_t)q * Mq + i) * qstride + (size_t)(kvh * p.n_rep + g) * DH;
-            rotate8(src + j0, src + j0 + half, p.rope + (size_t)pos * half + j0, p.qscale, lo, hi);
+            rotate8(src + j0, src + j0 + half, p.rope + (size_t)pos * half + j0, p.qscale, lo, hi, &rlo, &rhi);
         }
         *(uint4 *)(q_s + sw_off(qrows_pad, rr, j0)) = lo;
         *(uint4 *)(q_s + sw_off(qrows_pad, rr, j0 + half)) = hi;
+        *(uint4 *)(q_lo_s + sw_off(qrows_pad, rr, j0)) = rlo;
+        *(uint4 *)(q_lo_s + sw_off(qrows_pad, rr, j0 + half)) = rhi;
     }
     __syncthreads();
 
     WarpState<DH> w;
+    w.qlo_base = smem_u32(q_lo_s);
+    w.q_rows = qrows_pad;
+    w.q_row = mt * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
     if (compute) {
         const int row = mt * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
 #pragma unroll
@@ -702,7 +726,7 @@ int attention_tc(scd_session *s, int layer, int Mq, int pos_override, cudaStream
     // clusters of 7 take 1.8 times as long as clusters of 4 on the same problem)
     p.C = attention_clusters(s, plan);
     const int dh = c.head_dim;
-    const size_t q_bytes = ((size_t)p.n_mtiles * 16 * dh * 2 + 1023) & ~(size_t)1023;
+    const size_t q_bytes = 2 * (((size_t)p.n_mtiles * 16 * dh * 2 + 1023) & ~(size_t)1023);   // two planes
     const size_t stage_bytes = (size_t)2 * TK * dh * 2;
     const size_t merge_bytes = (size_t)p.n_mtiles * 16 * (dh + 2) * sizeof(float);
     // a ring deep enough to keep ~64 KB in flight per CTA, and wide enough for the merge staging

@@ -788,15 +788,16 @@ struct SessionGemm {                 // activation-side tensor maps of a session
     std::map<std::tuple<const void *, int, int>, CUtensorMap> xmaps;
 };
 
-// (both planes of an activation buffer in one map)
-int x_map(scd_session *s, const void *buf, int K, int nbox, CUtensorMap *out)
+// (planes = 2: both planes of an activation buffer in one map; 1: its hi plane alone)
+int x_map(scd_session *s, const void *buf, int K, int nbox, int planes, CUtensorMap *out)
 {
     SessionGemm *sg = (SessionGemm *)s->gemm_state;
-    auto key = std::make_tuple(buf, K, nbox);
+    auto key = std::make_tuple(buf, K, nbox * 4 + planes);
     auto it = sg->xmaps.find(key);
     if (it == sg->xmaps.end()) {
         CUtensorMap m;
-        int rc = make_map_planes(&m, buf, (uint64_t)s->rows_cap, (uint64_t)K, (uint32_t)nbox);
+        int rc = planes == 2 ? make_map_planes(&m, buf, (uint64_t)s->rows_cap, (uint64_t)K, (uint32_t)nbox)
+                             : make_map(&m, buf, (uint64_t)s->rows_cap, (uint64_t)K, (uint32_t)nbox);
         if (rc != SCD_OK) return rc;
         it = sg->xmaps.emplace(key, m).first;
     }
@@ -824,8 +825,10 @@ int w_map(GemmPlan *plan, const Segment &sg, int box_rows, CUtensorMap *out)
     return SCD_OK;
 }
 
+// x_planes: 2 = multiply with both planes of x, 1 = with its hi plane alone (where the output is rounded to
+// bf16 right away - Q, K, V - or is the last stage - the logits - the remainder plane buys nothing)
 int run_gemm(scd_session *s, int kind, const Segment *segs, int n_seg, int epi, const void *x, int K, int rows,
-             void *out, int ldo, const NormIn *nin, const NormOut *nout, cudaStream_t st)
+             void *out, int ldo, const NormIn *nin, const NormOut *nout, int x_planes, cudaStream_t st)
 {
     GemmPlan *plan = (GemmPlan *)s->model->gemm_plan;
     const bool pair = epi == EPI_SWIGLU;
@@ -848,7 +851,7 @@ int run_gemm(scd_session *s, int kind, const Segment *segs, int n_seg, int epi, 
     p.n_seg = pair ? 1 : n_seg;
     p.M = rows;
     p.nbox = round16(rows);
-    p.x_planes = 2;
+    p.x_planes = x_planes;
     p.out_plane = (long long)s->rows_cap * ldo;           // (used by the outputs that are GEMM inputs themselves)
     p.stages = choose_stages(p.nbox, p.x_planes, (p.k_blocks + p.k_splits - 1) / p.k_splits,
                              tiles * p.k_splits <= 2 * plan->sm_count, plan->forced_stages);
@@ -864,7 +867,7 @@ int run_gemm(scd_session *s, int kind, const Segment *segs, int n_seg, int epi, 
         SCD_REQUIRE(tiles <= s->ss_parts_cap, SCD_ERR_SHAPE, "norm statistics: %d tiles > %d", tiles, s->ss_parts_cap);
         p.gain_next = (const __nv_bfloat16 *)nout->gain; p.xg_out = (__nv_bfloat16 *)nout->xg; p.ss_out = nout->ss;
     }
-    int rc = x_map(s, x, K, p.nbox, &p.tmap_x);
+    int rc = x_map(s, x, K, p.nbox, p.x_planes, &p.tmap_x);
     if (rc != SCD_OK) return rc;
     p.err = (int *)s->gemm_ws;
     p.skip = s->skip_now;
@@ -906,7 +909,7 @@ int gemm_tc_qkv(scd_session *s, int l, int rows, int ss_parts, cudaStream_t st)
     const Segment segs[3] = {{m->wq[l], dq, d, 0, dq, 0}, {m->wk[l], dkv, d, 0, dkv, dq}, {m->wv[l], dkv, d, 0, dkv, dq + dkv}};
     const NormIn nin = {s->ss, ss_parts};
     // fp32 out: the attention kernel rotates Q and K in fp32 and rounds each of Q, K, V to bf16 once
-    return run_gemm(s, GEMM_QKV, segs, 3, EPI_F32, s->xn, d, rows, s->qkv, dq + 2 * dkv, &nin, nullptr, st);
+    return run_gemm(s, GEMM_QKV, segs, 3, EPI_F32, s->xn, d, rows, s->qkv, dq + 2 * dkv, &nin, nullptr, 1, st);
 }
 
 int gemm_tc_residual(scd_session *s, int l, int which, int rows, const void *gain_next, int *parts_out,
@@ -920,7 +923,7 @@ int gemm_tc_residual(scd_session *s, int l, int which, int rows, const void *gai
     const NormOut nout = {gain_next, s->xn, s->ss};
     const int rc = run_gemm(s, which == 0 ? GEMM_O : GEMM_DOWN, segs, 1, EPI_RESID, which == 0 ? s->att : s->act, K, rows,
                             s->h, c.d_model, nullptr,
-                            &nout, st);
+                            &nout, 2, st);
     *parts_out = g_last_tiles;                          // one partial sum of squares per output tile
     return rc;
 }
@@ -931,7 +934,7 @@ int gemm_tc_gate_up(scd_session *s, int l, int rows, int ss_parts, cudaStream_t 
     const scd_model_config_t &c = m->cfg;
     const Segment segs[2] = {{m->w_gate[l], c.d_ffn, c.d_model, 0, c.d_ffn, 0}, {m->w_up[l], c.d_ffn, c.d_model, 0, c.d_ffn, 0}};
     const NormIn nin = {s->ss, ss_parts};
-    return run_gemm(s, GEMM_GATE_UP, segs, 2, EPI_SWIGLU, s->xn, c.d_model, rows, s->act, c.d_ffn, &nin, nullptr, st);
+    return run_gemm(s, GEMM_GATE_UP, segs, 2, EPI_SWIGLU, s->xn, c.d_model, rows, s->act, c.d_ffn, &nin, nullptr, 2, st);
 }
 
 // Logits of the ids [lo, hi) and, when eol >= 0, of id eol; other columns of `logits` are left
@@ -946,7 +949,7 @@ int gemm_tc_lm_head(scd_session *s, int rows, float *logits, int lo, int hi, int
     if (eol >= 0 && !(eol >= lo8 && eol < hi))
         segs[n++] = {s->model->lm_head, c.vocab_out, c.d_model, eol & ~7, std::min(c.vocab_out, (eol & ~7) + 8), 0};
     const NormIn nin = {s->ss, ss_parts};
-    return run_gemm(s, GEMM_LM_HEAD, segs, n, EPI_F32, s->xn, c.d_model, rows, logits, c.vocab_out, &nin, nullptr, st);
+    return run_gemm(s, GEMM_LM_HEAD, segs, n, EPI_F32, s->xn, c.d_model, rows, logits, c.vocab_out, &nin, nullptr, 1, st);
 }
 
 void gemm_set_kind_splits(scd_model *m, int kind, int k_splits)
