@@ -27,17 +27,19 @@ if ROOT not in sys.path:
 METRIC = "generated_tokens_per_s"
 UNIT = "tokens/s"
 
+# Typed-in constants (NOT measured by a run of this file; each is labelled as such in the JSON line).
 # DRAM traffic of gemm_ws_kernel relative to its algorithmic (weight) bytes, from the ncu capture
-# summarised in profiles/gemm_ws_kernel_qkv_shape.md (dram__bytes_read.sum + dram__bytes_write.sum
-# = 104.7 MB for 100.66 MB of weights). Traffic grows in proportion to the weight bytes (every
-# weight is read once), so the figure is scaled to the average launch. Set to None when the
-# kernel changes until the counters are taken again.
-GEMM_TRAFFIC_RATIO = 1.040
+# summarised in profiles/gemm_ws_kernel_qkv_shape.md (dram__bytes_read.sum + dram__bytes_write.sum over
+# the weight bytes of that launch). Traffic grows in proportion to the weight bytes (every weight is read
+# once), so the ratio is applied to the average launch. None = the kernel changed since the capture.
+GEMM_TRAFFIC_RATIO = None
+GEMM_TRAFFIC_SOURCE = "profiles/gemm_ws_kernel_qkv_shape.md (ncu capture; typed in, not measured by this run)"
 
-# Tokens committed per forward on each workload, as measured by the CUDA arm (the oracle commits
-# the same tokens: parity). Used only to convert the oracle's seconds per iteration into tokens/s
-# in the reference arm, which cannot afford whole generations.
-MEASURED_ACCEPT = {"tiny": 1.6, "llamagen_xl": 4.8, "lumina_7b": 1.04, "video_4b": 1.02}
+# Tokens committed per forward on each workload, as measured by earlier runs of the CUDA arm (the oracle
+# commits the same tokens: parity). Used only by the reference arm, which cannot afford whole generations,
+# to convert the oracle's seconds per iteration into tokens/s.
+MEASURED_ACCEPT = {"tiny": 1.6, "llamagen_xl": 5.3, "lumina_7b": 1.05, "video_4b": 1.02, "janus_like": 1.05,
+                   "video_4b_top_p": 1.02}
 
 
 # ------------------------------------------------------------------------------------------ helpers
@@ -192,6 +194,8 @@ def oracle_sample(shape, weights_np, cond, uncond, n_layers_sample):
     for k in range(L):
         Wp[k], Zp[k] = oracle.postprocess(logits[0][k], logits[1][k] if S == 2 else None, lo, hi,
                                           shape["temperature"], shape["top_k"], shape["cfg_lambda"])
+        if shape.get("top_p", 0.0):
+            Wp[k], Zp[k] = oracle.top_p_filter(Wp[k], Zp[k], shape["top_p"])
         Wq[k], Zq[k] = oracle.uniform_weights(V, lo, hi)
     oracle.verify_window(Wp, Zp, Wq, Zq, drafts, P, 0, seed)
     return time.perf_counter() - t0
@@ -223,10 +227,11 @@ def run_reference(args, shape):
     # truncated model already carries in full; scale conservatively (all of it) by depth
     t_iter = float(np.mean(times)) * shape["n_layers"] / nl_s
     mean_a = args.assumed_accept if args.assumed_accept > 0 else MEASURED_ACCEPT.get(args.workload, 1.0)
+    accept_source = "--assumed-accept" if args.assumed_accept > 0 else "typed in from earlier runs of the CUDA arm"
     value = mean_a / t_iter
     sample = (f"one SCD iteration (S={S} x L={shape['window_L']} rows) of the {args.workload} shape on the first "
               f"{nl_s} of {shape['n_layers']} layers + full LM head + verify; time scaled by depth; tokens per "
-              f"forward {mean_a:.2f} (measured by the CUDA arm)")
+              f"forward {mean_a:.2f} ({accept_source})")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps_ref, "warmup": args.warmup_ref, "ms_per_step": t_iter * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64 accumulate over bf16 weights",
@@ -238,6 +243,21 @@ def run_reference(args, shape):
 
 
 # ------------------------------------------------------------------------------------------ CUDA arm
+def context_prompts(shape, cond, uncond, extra, seed=4321):
+    """The workload's prompt followed by `extra` synthetic generated-range ids (the same in both streams, as
+    generated tokens are): a stand-in for a generation that is `extra` tokens along, reached without
+    generating them. Forced end-of-row positions keep their id."""
+    if extra <= 0:
+        return cond, uncond
+    rng = np.random.default_rng(seed)
+    B = cond.shape[0]
+    gen = rng.integers(shape["allowed_lo"], shape["allowed_hi"], size=(B, extra)).astype(np.int32)
+    if shape["row_period"] > 0:
+        g = np.arange(extra)
+        gen[:, g % shape["row_period"] == shape["row_period"] - 1] = shape["eol_id"]
+    return np.concatenate([cond, gen], axis=1), np.concatenate([uncond, gen], axis=1)
+
+
 def run_scd(args, shape):
     import torch
     from paper_2510_24211_b200 import binding as scd
@@ -254,7 +274,8 @@ def run_scd(args, shape):
 
     B = args.batch
     S = 2 if shape["cfg_lambda"] != 0.0 else 1
-    L = shape["window_L"]
+    L = args.window if args.window > 0 else shape["window_L"]
+    shape = dict(shape, window_L=L)
     P, N = shape["prompt_len"], shape["n_gen"]
     max_seq = P + N + L
     w = synth.make_weights(shape, seed=1234, device="cuda")
@@ -262,19 +283,23 @@ def run_scd(args, shape):
     if args.gemm_splits or args.gemm_stages:
         model.scd_model_gemm_tune(args.gemm_splits, args.gemm_stages)
     cond, uncond = synth.make_prompt(shape, batch=B)
-    prompts = np.concatenate([cond, uncond]) if S == 2 else cond
 
     def cfg_of(mode):
         return scd.decode_config(mode=mode, batch=B, window_L=L, temperature=shape["temperature"],
                                  top_k=shape["top_k"], cfg_lambda=shape["cfg_lambda"], seed=shape["seed"] + rank,
                                  allowed_lo=shape["allowed_lo"], allowed_hi=shape["allowed_hi"],
-                                 row_period=shape["row_period"], eol_id=shape["eol_id"], alpha=args.alpha)
+                                 row_period=shape["row_period"], eol_id=shape["eol_id"], alpha=args.alpha,
+                                 top_p=shape.get("top_p", 0.0))
 
     coupling = {"scd_mc": scd.SCD_MODE_SCD_MC, "scd_gs": scd.SCD_MODE_SCD_GS, "sjd": scd.SCD_MODE_SJD,
                 "alpha": scd.SCD_MODE_ALPHA}[args.coupling]
     sess = scd.Session(model, cfg_of(coupling))
     tuned = None
     stream = torch.cuda.current_stream()
+    peaks = measured_peaks()
+    wb = weight_bytes(shape)
+    gemm_classes = ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_head")
+    gemm_bytes = sum(wb[c] for c in gemm_classes)
 
     def barrier():
         torch.cuda.synchronize()
@@ -282,55 +307,84 @@ def run_scd(args, shape):
             dist.barrier()
             torch.cuda.synchronize()
 
+    def prefill_at(extra):
+        """A generation `extra` tokens along: the remaining N - extra tokens are still to come."""
+        c, u = context_prompts(shape, cond, uncond, extra)
+        sess.scd_prefill(np.concatenate([c, u]) if S == 2 else c, n_new=N - extra)
+        return P + extra
+
+    def timed_steps(steps, extra):
+        """Exactly `steps` iterations (CUDA events on the launching stream), in segments that never run past
+        the end of a generation; a generation that ends is restarted (untimed) at the same context."""
+        n_total = P + N
+        done, tokens, total_ms, ctx_sum = 0, 0, 0.0, 0.0
+        _, n_now, _ = sess.scd_step_result()
+        while done < steps:
+            remaining = int((n_total - n_now).max())
+            if remaining <= 0:
+                prefill_at(extra)                            # untimed: a new generation starts
+                _, n_now, _ = sess.scd_step_result()
+                continue
+            seg = min(steps - done, (remaining + L - 1) // L)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(seg):
+                sess.scd_step()
+            e1.record(stream)
+            e1.synchronize()
+            total_ms += e0.elapsed_time(e1)
+            _, n_after, _ = sess.scd_step_result()
+            tokens += int((n_after - n_now).sum())
+            ctx_sum += seg * float(n_now.mean() + n_after.mean()) / 2.0
+            n_now = n_after
+            done += seg
+        return total_ms, tokens, ctx_sum / max(done, 1)
+
+    def step_bytes_at(mean_ctx):
+        # whole iteration: weights + KV read at the mean context of the timed region + verify rows
+        return gemm_bytes + mean_ctx * S * B * kv_bytes_per_token(shape) + verify_bytes(shape, B, S, L)
+
     # ---- warm-up: a fresh generation, W steps -----------------------------------------------------
-    sess.scd_prefill(prompts, n_new=N)
+    start_extra = {"start": 0, "mid": N // 2, "end": max(0, N - 2 * L)}[args.context]
+    prefill_at(start_extra)
     if args.autotune:
         tuned = [int(x) for x in sess.scd_autotune()]
     for _ in range(max(args.warmup, 3)):
         sess.scd_step()
     torch.cuda.synchronize()
 
-    # ---- timed: exactly K steps, in segments that never run past the end of a generation ----------
-    n_total = P + N
+    # ---- timed: exactly K steps ------------------------------------------------------------------
     sampler = ClockSampler(local)
     launches0 = scd.scd_kernel_launches()
     barrier()
     sampler.start()
-    done, tokens, total_ms, ctx_sum = 0, 0, 0.0, 0.0
-    _, n_now, _ = sess.scd_step_result()
-    while done < args.steps:
-        remaining = int((n_total - n_now).max())
-        if remaining <= 0:
-            sess.scd_prefill(prompts, n_new=N)           # untimed: a new generation starts
-            _, n_now, _ = sess.scd_step_result()
-            continue
-        seg = min(args.steps - done, (remaining + L - 1) // L)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(seg):
-            sess.scd_step()
-        e1.record(stream)
-        e1.synchronize()
-        total_ms += e0.elapsed_time(e1)
-        _, n_after, _ = sess.scd_step_result()
-        tokens += int((n_after - n_now).sum())
-        ctx_sum += seg * float(n_now.mean() + n_after.mean()) / 2.0
-        n_now = n_after
-        done += seg
+    total_ms, tokens, mean_ctx = timed_steps(args.steps, start_extra)
     barrier()
     clocks = sampler.stop()
     launches = scd.scd_kernel_launches() - launches0
-    mean_ctx = ctx_sum / max(done, 1)
 
     total_ms_all, tokens_all = aggregate_over_ranks(total_ms, tokens, world, "cuda")
     value = tokens_all / (total_ms_all * 1e-3)
     ms_per_step = total_ms_all / args.steps
     accepted_per_forward = tokens / (args.steps * B)
 
+    # ---- the same iteration at the start, the middle and the end of the context --------------------
+    by_context = {}
+    if world == 1 and not args.no_contexts:
+        for name, extra in (("start", 0), ("mid", N // 2), ("end", max(0, N - 2 * L))):
+            prefill_at(extra)
+            for _ in range(3):
+                sess.scd_step()
+            torch.cuda.synchronize()
+            ms, _, ctx = timed_steps(args.context_steps, extra)
+            msps = ms / args.context_steps
+            by_context[name] = {"context_tokens": ctx, "ms_per_step": msps, "bytes_per_step": step_bytes_at(ctx),
+                                "step_roofline_frac": step_bytes_at(ctx) / (msps * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+
     # ---- per-kernel attribution of an iteration (device events in front of every kernel) ----------
     prof_ms = np.zeros(len(scd.PROF_CLASSES), dtype=np.float32)
     prof_n = np.zeros(len(scd.PROF_CLASSES), dtype=np.int32)
-    sess.scd_prefill(prompts, n_new=N)
+    prefill_at(start_extra)
     for _ in range(3):
         sess.scd_step()
     n_prof = 0
@@ -343,57 +397,54 @@ def run_scd(args, shape):
     tl_n = np.zeros(len(scd.PROF_CLASSES), dtype=np.int32)
     for _ in range(args.profile_steps):
         sess.scd_step_timeline(tl_ms, tl_n)
-    peaks = measured_peaks()
-    wb = weight_bytes(shape)
-    rows = S * B * L
     by_class = {c: float(prof_ms[i]) / max(n_prof, 1) for i, c in enumerate(scd.PROF_CLASSES)}
     launches_by_class = {c: int(prof_n[i]) // max(n_prof, 1) for i, c in enumerate(scd.PROF_CLASSES)}
-    gemm_classes = ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_head")
-    gemm_ms_isolated = sum(by_class[c] for c in gemm_classes)
+    gemm_ms_events = sum(by_class[c] for c in gemm_classes)
     gemm_launches = sum(launches_by_class[c] for c in gemm_classes)
-    gemm_bytes = sum(wb[c] for c in gemm_classes)
     timeline = {c: float(tl_ms[i]) / max(n_prof, 1) for i, c in enumerate(scd.PROF_CLASSES)}
-    gemm_ms = sum(timeline[c] for c in gemm_classes)
+    gemm_ms_inflight = sum(timeline[c] for c in gemm_classes)
     roofline = None
-    if gemm_launches > 0 and gemm_ms > 0:
-        achieved = gemm_bytes / (gemm_ms * 1e-3) / 1e9
-        isolated = gemm_bytes / (gemm_ms_isolated * 1e-3) / 1e9 if gemm_ms_isolated > 0 else None
+    if gemm_launches > 0 and gemm_ms_events > 0:
+        # headline: every launch timed on its own by CUDA events (the conservative figure: events between
+        # the kernels switch their programmatic overlap off); second: the kernels as they overlap in a step
+        achieved = gemm_bytes / (gemm_ms_events * 1e-3) / 1e9
+        inflight = gemm_bytes / (gemm_ms_inflight * 1e-3) / 1e9 if gemm_ms_inflight > 0 else None
         roofline = {"bound": "hbm", "kernel": "gemm_ws_kernel (all weight GEMMs of an iteration)",
                     "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                    "timing": "device time stamps inside the kernels (completion to completion, kernels "
-                              "overlapping as in the timed region)",
+                    "timing": "CUDA events on the launching stream around every launch (no overlap between kernels)",
                     "bytes_per_launch": gemm_bytes / gemm_launches,
-                    "us_per_launch": gemm_ms * 1e3 / gemm_launches, "launches_per_step": gemm_launches,
-                    "achieved_isolated": isolated,
-                    "frac_isolated": isolated / peaks["hbm_gbs"] if isolated else None,
-                    "us_per_launch_isolated": gemm_ms_isolated * 1e3 / gemm_launches,
-                    "isolated_note": "CUDA events between the kernels: every launch timed on its own, no overlap",
+                    "us_per_launch": gemm_ms_events * 1e3 / gemm_launches, "launches_per_step": gemm_launches,
+                    "achieved_inflight": inflight,
+                    "frac_inflight": inflight / peaks["hbm_gbs"] if inflight else None,
+                    "us_per_launch_inflight": gemm_ms_inflight * 1e3 / gemm_launches,
+                    "inflight_note": "device time stamps inside the kernels, completion to completion, kernels "
+                                     "overlapping (programmatic dependent launch) as in the timed region",
                     "traffic": (gemm_bytes / gemm_launches) * GEMM_TRAFFIC_RATIO if GEMM_TRAFFIC_RATIO else None,
-                    "traffic_note": "bytes per average launch; ncu counters of the QKV-shaped launch scaled by weight bytes"}
-    # whole iteration: weights + KV read at the mean context of the timed region + verify rows
-    step_bytes = gemm_bytes + mean_ctx * S * B * kv_bytes_per_token(shape) + verify_bytes(shape, B, S, L)
+                    "traffic_source": GEMM_TRAFFIC_SOURCE}
+    step_bytes = step_bytes_at(mean_ctx)
     step_roofline = {"bound": "hbm", "achieved": step_bytes / (ms_per_step * 1e-3) / 1e9 if world == 1 else None,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "bytes_per_step": step_bytes,
                      "mean_context_tokens": mean_ctx}
     if step_roofline["achieved"]:
         step_roofline["frac"] = step_roofline["achieved"] / peaks["hbm_gbs"]
-    # the fused verify kernel: by bytes it belongs to the HBM roofline, in practice it is bound by
-    # instruction issue (see profiles/); reported so that the gap is visible, timed on its own
+    # the fused verify kernel: by bytes it belongs to the HBM roofline, in practice it is bound by the
+    # latency of its chain of row-wide exchanges (see profiles/); reported so that the gap is visible
     verify_roofline = None
     if by_class.get("verify", 0.0) > 0:
         vb = verify_bytes(shape, B, S, L)
         vach = vb / (by_class["verify"] * 1e-3) / 1e9
-        verify_roofline = {"bound": "hbm", "kernel": "verify_kernel", "achieved": vach, "peak": peaks["hbm_gbs"],
+        verify_roofline = {"bound": "hbm", "kernel": "verify kernel", "achieved": vach, "peak": peaks["hbm_gbs"],
                            "unit": "GB/s", "frac": vach / peaks["hbm_gbs"], "bytes_per_launch": vb,
                            "us_per_launch": by_class["verify"] * 1e3,
-                           "note": "instruction-issue bound: 48 % issue utilisation on the SMs it occupies"}
+                           "timing": "CUDA events around the launch (includes the launch gap)"}
 
     # ---- the same library's vanilla AR path (speed-up denominator) --------------------------------
     ar_ms, ar_tokens_per_s = None, None
     if not args.no_ar:
         ar = scd.Session(model, cfg_of(scd.SCD_MODE_AR))
-        ar.scd_prefill(prompts, n_new=N)
+        c, u = context_prompts(shape, cond, uncond, start_extra)
+        ar.scd_prefill(np.concatenate([c, u]) if S == 2 else c, n_new=N - start_extra)
         for _ in range(3):
             ar.scd_step()
         torch.cuda.synchronize()
@@ -410,6 +461,7 @@ def run_scd(args, shape):
     # ---- end to end through the public calls: host prompt in, host tokens out ---------------------
     e2e = None
     if not args.no_e2e:
+        prompts = np.concatenate([cond, uncond]) if S == 2 else cond
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         sess.scd_prefill(prompts, n_new=N)
@@ -423,19 +475,22 @@ def run_scd(args, shape):
         e2e = {"value": e2e_value, "unit": UNIT,
                "what": "scd_prefill(host prompt) + scd_generate(host tokens out), wall clock, whole generation",
                "forwards": int(st.forwards), "accepted_per_forward": N / fw, "seconds": e2e_s,
+               "ms_per_forward": e2e_s * 1e3 / fw,
                "h2d_bytes_per_step": prompts.nbytes / fw, "d2h_bytes_per_step": toks.nbytes / fw}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if shape["dtype"] == "bf16" else "f32",
             "data": "synthetic",
-            "config": config_of(args, shape),
+            "config": dict(config_of(args, shape), context=args.context),
             "accepted_tokens_per_forward": accepted_per_forward,
             "speedup_vs_own_ar": (value / world / ar_tokens_per_s) if ar_tokens_per_s else None,
             "ar_tokens_per_s": ar_tokens_per_s,
             "ar_ms_per_step": ar_ms,
+            "scd_step_over_ar_step": (ms_per_step / ar_ms) if ar_ms else None,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
             "roofline": roofline, "step_roofline": step_roofline, "verify_roofline": verify_roofline,
+            "by_context": by_context,
             "autotuned_k_splits": tuned,
             "ms_by_kernel_class": {c: round(v, 5) for c, v in by_class.items() if v > 0},
             "ms_by_kernel_class_overlapped": {c: round(v, 5) for c, v in timeline.items() if v > 0}}
@@ -444,7 +499,6 @@ def run_scd(args, shape):
     if world == 1 and not args.no_cpu_baseline:
         cores = os.cpu_count() or 1
         nl_s = min(shape["n_layers"], args.ref_layers)
-        sub = dict(shape, n_layers=nl_s)
         keep = ("tok_emb", "final_norm", "lm_head")
         wn = {k: synth.to_numpy(w[k]) for k in keep}
         for k in synth.LAYER_KEYS:
@@ -487,6 +541,11 @@ def main():
     ap.add_argument("--gemm-stages", type=int, default=0, help="tuning: force the ring depth of every GEMM (0 = automatic)")
     ap.add_argument("--no-ar", action="store_true", help="skip the vanilla-AR arm (short profiling runs)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end arm (short profiling runs)")
+    ap.add_argument("--context", choices=("start", "mid", "end"), default="start",
+                    help="where in the generation the timed region starts (a synthetic prompt of that length is prefilled)")
+    ap.add_argument("--no-contexts", action="store_true", help="skip the start / mid / end measurements")
+    ap.add_argument("--context-steps", type=int, default=24, help="iterations timed at each of start / mid / end")
+    ap.add_argument("--window", type=int, default=0, help="Jacobi window L (0 = the workload's)")
     args = ap.parse_args()
     from paper_2510_24211_b200 import synth
     shape = dict(synth.WORKLOADS[args.workload])

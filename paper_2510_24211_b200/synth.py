@@ -36,6 +36,18 @@ WORKLOADS = {
         vocab_out=64000, vocab_in=64000, dtype="bf16", rope_base=10000.0, rms_eps=1e-5,
         prompt_len=2560, n_gen=10240, window_L=64, temperature=1.0, top_k=1000, cfg_lambda=0.0,
         allowed_lo=0, allowed_hi=64000, row_period=0, eol_id=0, seed=0),
+    # the paper's Janus-Pro setting on a 7B-shaped decoder: 24 x 24 image tokens, guidance 5, top-k 1000
+    "janus_like": dict(
+        n_layers=30, d_model=4096, n_heads=32, n_kv_heads=32, head_dim=128, d_ffn=11008,
+        vocab_out=16384, vocab_in=16384 + 1024, dtype="bf16", rope_base=10000.0, rms_eps=1e-5,
+        prompt_len=64, n_gen=576, window_L=32, temperature=1.0, top_k=1000, cfg_lambda=5.0,
+        allowed_lo=0, allowed_hi=16384, row_period=0, eol_id=0, seed=0),
+    # the paper's video setting on the video-shaped decoder: nucleus 0.8, no top-k
+    "video_4b_top_p": dict(
+        n_layers=28, d_model=3072, n_heads=24, n_kv_heads=24, head_dim=128, d_ffn=8192,
+        vocab_out=64000, vocab_in=64000, dtype="bf16", rope_base=10000.0, rms_eps=1e-5,
+        prompt_len=2560, n_gen=10240, window_L=64, temperature=1.0, top_k=0, top_p=0.8, cfg_lambda=0.0,
+        allowed_lo=0, allowed_hi=64000, row_period=0, eol_id=0, seed=0),
 }
 
 LAYER_KEYS = ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down")

@@ -193,3 +193,15 @@ def test_generated_sequences_follow_the_exact_ar_joint(mode, L):
         dof += 1
     assert dof >= 20
     assert chi2 < dof + 4.5 * math.sqrt(2 * dof), (chi2, dof)
+
+
+# ---- the paper's other two settings as workloads (reduced depth) -------------------------------------------
+@pytest.mark.parametrize("name", ["janus_like", "video_4b_top_p"])
+def test_step_replay_paper_settings_reduced_depth(name):
+    """Janus-Pro-like (guidance 5, top-k 1000, 24 x 24 tokens) and the video setting with nucleus 0.8 and no
+    top-k (App. "Experimental Details"), on two layers of the workload's shape: every decision of a short
+    generation replayed through the oracle's loop."""
+    w = synth.WORKLOADS[name]
+    shape = dict(w, n_layers=2)
+    _replay_case(shape, oracle.MODE_SCD_MC, B=1, L=w["window_L"], P=6, n_new=70, top_k=w["top_k"], lam=w["cfg_lambda"],
+                 seed=19, lo=w["allowed_lo"], hi=w["allowed_hi"], std=0.02, page=64, top_p=w.get("top_p", 0.0))
