@@ -458,6 +458,23 @@ def run_scd(args, shape):
         ar_tokens_per_s = B / (ar_ms * 1e-3)
         ar.close()
 
+    # ---- prefill of the workload's prompt (compute-bound for long prompts) ------------------------
+    prefill = None
+    if world == 1:
+        prompts0 = np.concatenate([cond, uncond]) if S == 2 else cond
+        sess.scd_prefill(prompts0, n_new=N)              # warm (tensor maps, kernels)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        sess.scd_prefill(prompts0, n_new=N)
+        torch.cuda.synchronize()
+        pf_s = time.perf_counter() - t0
+        params = sum(wb[c] for c in ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down")) / (4 if shape["dtype"] == "f32" else 2)
+        flops = 2.0 * params * S * B * max(P - 1, 0)
+        prefill = {"prompt_tokens": P, "streams": S * B, "ms": pf_s * 1e3, "timing": "wall clock around scd_prefill (host copy in, synchronised)",
+                   "tflops": flops / pf_s / 1e12 if pf_s > 0 else None,
+                   "frac_of_bf16_sustained": flops / pf_s / 1e12 / peaks["bf16_tflops_sustained"] if pf_s > 0 else None,
+                   "flops_note": "2 x layer parameters x prompt rows (attention and the second activation plane not counted)"}
+
     # ---- end to end through the public calls: host prompt in, host tokens out ---------------------
     e2e = None
     if not args.no_e2e:
@@ -490,7 +507,7 @@ def run_scd(args, shape):
             "scd_step_over_ar_step": (ms_per_step / ar_ms) if ar_ms else None,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
             "roofline": roofline, "step_roofline": step_roofline, "verify_roofline": verify_roofline,
-            "by_context": by_context,
+            "by_context": by_context, "prefill": prefill,
             "autotuned_k_splits": tuned,
             "ms_by_kernel_class": {c: round(v, 5) for c, v in by_class.items() if v > 0},
             "ms_by_kernel_class_overlapped": {c: round(v, 5) for c, v in timeline.items() if v > 0}}

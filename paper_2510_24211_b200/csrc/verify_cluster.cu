@@ -7,18 +7,27 @@
 //
 // Passes over a row (all on registers; the only HBM traffic is the logits in, the draft weights in and,
 // in a session, the target weights out):
-//   1. x = post-processed logit (guidance mix, temperature); row maximum m          -> barrier 1
-//   2. histogram of the LIVE ids (x >= m - 22: only they can get a non-zero weight) over 2048 equal
-//      steps of m - x; merged by every CTA; the step holding the k-th largest        -> barrier 2
-//   3. the ids of that step go to a short list; every CTA reads all lists and picks the exact k-th
-//      largest by counting (radix selection over the cluster when the lists overflow) -> barrier 3
-//   4. integer weights W = trunc(scd_exp(x - m) 2^30) for x >= tau, their sum Z       -> barrier 4
-//      accept test of Algorithm 1 in 128-bit integers (computed alike by every CTA)
-//   5. on rejection: residual mass R_v = max(0, Wp_v Zq - Wq_v Zp) per CTA            -> barrier 5
+//   1. x = post-processed logit (guidance mix, temperature); row maximum m                -> barrier 1
+//   2. W = trunc(scd_exp(x - m) 2^30) for every LIVE id (x >= m - 22: only they can get a non-zero
+//      weight) and a histogram of the live ids over 512 equal steps of m - x; every CTA merges the
+//      histograms and finds the step that holds the k-th largest                           -> barrier 2
+//   3. mass of the ids above that step, summed per CTA; the ids OF the step go to a short list as
+//      (key of x, W); every CTA reads all lists, picks the exact k-th largest by counting (radix
+//      selection over the cluster when the lists overflow) and has the normaliser:
+//      Z = mass above the step + the candidates that stay; ids below tau lose their weight -> barrier 3
+//      accept test of Algorithm 1 in 128-bit integers, computed alike by every CTA (each weighs the draft
+//      itself, from the draft's own logits)
+//   4. on rejection: residual mass R_v = max(0, Wp_v Zq - Wq_v Zp) per CTA                 -> barrier 4
 //      and the inverse-CDF walk inside the one warp that holds the target
-// A stand-alone call with raw draft logits runs passes 1-4 on both rows at once. The CTA that finishes
-// a row takes the sequence's ticket; the last ticket of a sequence does the only serial part (first
-// rejection, commit, next window), exactly as in the one-CTA-per-row kernel.
+// A stand-alone call with raw draft logits runs passes 1-3 on both rows at once. The CTA that finds a
+// row's token writes it and takes the sequence's ticket (with two tokens per row - SJD, alpha - rank 0
+// does, after the closing barrier); the last ticket of a sequence does the only serial part (first
+// rejection, commit, next window), exactly as in the one-CTA-per-row kernel. The closing barrier (nobody
+// may leave while a peer still reads its shared memory) is off the critical path: everybody arrives as
+// soon as it has finished reading, the ticket's CTA waits only at its very end.
+//
+// What every thread needs from every peer (maxima, masses, counts) is fetched by ONE lane per peer and
+// handed on through local shared memory: distributed shared memory is for few, wide requests.
 //
 // Fewer than top_k live ids: the k-th largest then has weight 0 and so has everything below it, so
 // the threshold is dropped - the weights are those of the definition.

@@ -217,6 +217,11 @@ def test_step_replay_wide_window_ragged_batch_bf16():
     _replay_case(MID_BF16_D64, oracle.MODE_SCD_MC, B=3, L=48, P=66, n_new=120, top_k=60, seed=17, page=64)
 
 
+def test_step_replay_four_cfg_pairs_fill_the_row_limit():
+    # B = 4 with guidance at L = 32: 256 window rows in one forward, the most a bf16 session carries
+    _replay_case(MID_BF16_D64, oracle.MODE_SCD_MC, B=4, L=32, P=40, n_new=70, top_k=40, lam=1.5, seed=23, page=64)
+
+
 def test_autotune_keeps_state_and_parity():
     # the K slicing chosen by timing changes launch shapes only: decisions still replay through the oracle
     _replay_case(MID_BF16_D64, oracle.MODE_SCD_MC, B=2, L=16, P=70, n_new=60, top_k=40, lam=2.0, seed=19,
