@@ -42,8 +42,7 @@ namespace scd {
 
 namespace {
 
-constexpr int CT = 512;            // threads per CTA
-constexpr int CNW = CT / 32;
+constexpr int MAXW = 32;           // warps per CTA at most (512 or 1024 threads)
 constexpr int NB = 512;            // steps of the live range in the top-k histogram
 constexpr int CAND_CAP = 512;      // candidates one CTA may hand over
 constexpr int CAND_ALL = 1024;     // candidates of a whole row that are selected by counting
@@ -60,6 +59,10 @@ struct Xchg {                      // read by the peers through distributed shar
     unsigned hist[2][NB];          // (first: read with 16-byte loads)
     uint2 cand[2][CAND_CAP];       // (order-preserving key of x, weight) of the ids in the selected step
     unsigned radix[1024];          // overflow path: four passes x 256 counters
+    // nucleus threshold: mass per byte value of the weight, one table per pass, as two 32-bit sums (low 15 bits
+    // of the weights / the rest: a row has at most 2^16 ids and a weight 30 bits, so neither overflows) -
+    // 32-bit shared-memory adds stay fast when a flat distribution sends thousands of ids to one value
+    unsigned massh[4][2][256];
     unsigned long long zpart[2];   // mass of this CTA's ids above the selected step (overflow path: above the threshold)
     unsigned long long res_lo, res_hi;   // residual mass of this CTA's slice (two limbs)
     float mx[2];
@@ -67,8 +70,8 @@ struct Xchg {                      // read by the peers through distributed shar
 };
 
 struct Local {
-    float red_f[2][CNW];
-    unsigned long long red_u[2][CNW];
+    float red_f[2][MAXW];
+    unsigned long long red_u[2][MAXW];
     unsigned scan_w[2][4];
     int sel_bucket[2];
     unsigned sel_k[2];
@@ -78,7 +81,10 @@ struct Local {
     unsigned long long pz[2][MAXC], pr[2][MAXC];
     unsigned pc[2][MAXC];
     unsigned tau_key[2];
-    unsigned long long w_lo[CNW], w_hi[CNW];   // per-warp sums of a search (two limbs)
+    unsigned long long w_lo[MAXW], w_hi[MAXW];   // per-warp sums of a search (two limbs)
+    unsigned long long merged[256];            // nucleus threshold: the cluster's mass per byte value
+    unsigned long long np_above, np_kept;
+    unsigned np_sel;
     int last;
     int result;
 };
@@ -177,9 +183,10 @@ __device__ __forceinline__ int walk_slice(const unsigned (&wp)[EPT], const unsig
     return found < hi ? found : -1;
 }
 
-template <int EPT>
-__global__ void __launch_bounds__(CT, EPT <= 8 ? 2 : 1) verify_cluster_kernel(const VerifyParams p, int C)
+template <int EPT, int CT>
+__global__ void __launch_bounds__(CT, (CT == 512 && EPT <= 8) ? 2 : 1) verify_cluster_kernel(const VerifyParams p, int C)
 {
+    constexpr int CNW = CT / 32;
     __shared__ __align__(16) Xchg xc;
     __shared__ Local lc;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -521,14 +528,111 @@ __global__ void __launch_bounds__(CT, EPT <= 8 ? 2 : 1) verify_cluster_kernel(co
         });
         // the threshold takes effect: ids below it lose their weight (the step is monotone in x, so this
         // removes exactly the ids of later steps and the candidates below tau)
-        {
-            unsigned *wstore = p.keep_x ? (unsigned *)(p.xbuf[w.parity] + row * V) : nullptr;
+#pragma unroll
+        for (int i = 0; i < EPT; ++i) {
+            if (!(xv[0][i] >= tau[0])) wt[0][i] = 0u;
+            if (rawq && !(xv[1][i] >= tau[1])) wt[1][i] = 0u;
+        }
+        // ---- nucleus (top-p) on the integer weights: theta = the largest weight value whose ids {W >= theta}
+        // hold at least top_p of the mass; radix descent over the weight value, 8 bits per pass, with the
+        // MASS per byte value merged over the cluster (integers: the same theta in every CTA)
+        unsigned theta[2] = {0u, 0u};
+        if (p.top_p24) {
+            for (int i = tid; i < 4 * 2 * 256; i += CT) (&xc.massh[0][0][0])[i] = 0u;
+            EACH_ARRAY([&](auto A_) {
+                constexpr int a = decltype(A_)::value;
+                const u128 need = (u128)p.top_p24 * Zall[a];
+                unsigned prefix = 0, mask = 0;
+                unsigned long long above = 0, kept = 0;
+                __syncthreads();         // the tables are zeroed
+                for (int pass = 0; pass < 4; ++pass) {
+                    const int shift = 24 - 8 * pass;
+#pragma unroll
+                    for (int i = 0; i < EPT; ++i) {
+                        const unsigned wv = wt[a][i];
+                        if (wv != 0u && (wv & mask) == prefix) {
+                            const unsigned bin = (wv >> shift) & 255u;
+                            atomicAdd(&xc.massh[pass][0][bin], wv & 0x7FFFu);
+                            atomicAdd(&xc.massh[pass][1][bin], wv >> 15);
+                        }
+                    }
+                    cluster_sync();
+                    if (tid < 256) {
+                        unsigned long long mm = 0;
+                        for (int r = 0; r < C; ++r)
+                            mm += ((unsigned long long)ld_peer_u32(&xc.massh[pass][1][tid], (uint32_t)r) << 15) +
+                                  ld_peer_u32(&xc.massh[pass][0][tid], (uint32_t)r);
+                        lc.merged[tid] = mm;
+                    }
+                    __syncthreads();
+                    if (warp == 0) {
+                        // the highest byte value at which the mass from the top reaches `need`: lane l owns the
+                        // values 8 l .. 8 l + 7; suffix sums over the lanes, then each lane walks its eight
+                        unsigned long long mine8 = 0;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) mine8 += lc.merged[8 * lane + j];
+                        unsigned long long suf = mine8;              // sum over lanes >= lane
+#pragma unroll
+                        for (int o = 1; o < 32; o <<= 1) {
+                            const unsigned long long t = __shfl_down_sync(FULLM, suf, o);
+                            if (lane + o < 32) suf += t;
+                        }
+                        unsigned long long cum = above + suf - mine8;   // mass above my eight values
+                        int sel = -1;
+                        unsigned long long cum_at = 0, mass_at = 0;
+#pragma unroll
+                        for (int j = 7; j >= 0; --j) {
+                            const unsigned long long mb = lc.merged[8 * lane + j];
+                            if (sel < 0 && mb != 0ull && (((u128)(cum + mb) << 24) >= need)) { sel = 8 * lane + j; cum_at = cum; mass_at = mb; }
+                            cum += mb;
+                        }
+                        const unsigned hit = __ballot_sync(FULLM, sel >= 0);
+                        // (the total reaches `need` by construction, so some lane has a hit; the highest one wins)
+                        if (hit != 0u && lane == 31 - __clz(hit)) { lc.np_sel = (unsigned)sel; lc.np_above = cum_at; lc.np_kept = cum_at + mass_at; }
+                        if (hit == 0u && lane == 0) { lc.np_sel = 0u; lc.np_above = above; lc.np_kept = above; }
+                    }
+                    __syncthreads();
+                    prefix |= lc.np_sel << shift;
+                    mask |= 0xFFu << shift;
+                    above = lc.np_above;
+                    kept = lc.np_kept;
+                    __syncthreads();
+                }
+                theta[a] = prefix;
+                Zall[a] = kept;
+                unsigned long long z = 0;
+#pragma unroll
+                for (int i = 0; i < EPT; ++i) {
+                    if (wt[a][i] < prefix) wt[a][i] = 0u;
+                    z += wt[a][i];
+                }
+                // the slices' masses after the cut (an independent draw walks them in id order)
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(FULLM, z, o);
+                if (lane == 0) lc.red_u[a][warp] = z;
+                __syncthreads();
+                if (tid == 0) {
+                    unsigned long long t = 0;
+                    for (int i = 0; i < CNW; ++i) t += lc.red_u[a][i];
+                    xc.zpart[a] = t;
+                }
+                cluster_sync();          // the masses are published; every peer has finished reading my tables
+                if (a == 0) {
+                    if (warp == 0 && lane < MAXC) lc.pz[0][lane] = lane < C ? ld_peer_u64(&xc.zpart[0], (uint32_t)lane) : 0ull;
+                    __syncthreads();
+                    Zbefore[0] = 0;
+                    for (int r = 0; r < rank; ++r) Zbefore[0] += lc.pz[0][r];
+                    if (rawq)            // the draft row uses the tables next
+                        for (int i = tid; i < 4 * 2 * 256; i += CT) (&xc.massh[0][0][0])[i] = 0u;
+                }
+            });
+        }
+        if (p.keep_x) {
+            unsigned *wstore = (unsigned *)(p.xbuf[w.parity] + row * V);
 #pragma unroll
             for (int i = 0; i < EPT; ++i) {
                 const int v = wbase + 32 * i + lane;
-                if (!(xv[0][i] >= tau[0])) wt[0][i] = 0u;
-                if (rawq && !(xv[1][i] >= tau[1])) wt[1][i] = 0u;
-                if (wstore && v < hi) wstore[v] = wt[0][i];
+                if (v < hi) wstore[v] = wt[0][i];
             }
         }
         const unsigned long long Zp = Zall[0];
@@ -537,15 +641,15 @@ __global__ void __launch_bounds__(CT, EPT <= 8 ? 2 : 1) verify_cluster_kernel(co
         else if (fresh) Zq = (unsigned long long)(hi - lo);
         else Zq = Zq_stored;
         if (rank == 0 && tid == 0) {
-            RowStats st; st.m = m[0]; st.tau = tau[0]; st.Z = Zp; st.theta = 0u; st.pad_ = 0u;
+            RowStats st; st.m = m[0]; st.tau = tau[0]; st.Z = Zp; st.theta = theta[0]; st.pad_ = 0u;
             p.stats[w.parity][row] = st;
         }
 
         // ---- Algorithm 1 on (p, q, X) ------------------------------------------------------------------
         int accept = 1;
         if (mrs) {
-            const unsigned WpX = x_in ? weight_of(xX, m[0], tau[0]) : 0u;
-            const unsigned WqX = !x_in ? 0u : rawq ? weight_of(xqX, m[1], tau[1]) : fresh ? 1u : __float_as_uint(xqX);
+            const unsigned WpX = x_in ? weight_of(xX, m[0], tau[0], theta[0]) : 0u;
+            const unsigned WqX = !x_in ? 0u : rawq ? weight_of(xqX, m[1], tau[1], theta[1]) : fresh ? 1u : __float_as_uint(xqX);
             const unsigned Ua = noise_u24(p.seed, NOISE_ACCEPT, (unsigned)b, pos, w.t, 0);
             // u <= min(1, p(X)/q(X)) with u = (Ua+1)/2^24  <=>  (Ua+1) Wq[X] Zp <= Wp[X] Zq 2^24;
             // a draft without mass under p is rejected
@@ -708,20 +812,20 @@ __global__ void __launch_bounds__(CT, EPT <= 8 ? 2 : 1) verify_cluster_kernel(co
     }
 }
 
-// cluster size and ids per thread for rows of at most n ids, `rows` rows in the grid
-bool choose_cluster(int n, int rows, int sm_count, int *C_out, int *ept_out)
+// cluster size, threads per CTA and ids per thread for rows of at most n ids, `rows` rows in the grid
+bool choose_cluster(int n, int rows, int sm_count, int *C_out, int *ept_out, int *ct_out)
 {
     int C = 1;
     while (C < MAXC && rows * C * 2 <= sm_count) C *= 2;              // at most one CTA per SM (two would share its issue slots)
-    while (C > 1 && (C / 2) * 4 * CT >= n) C /= 2;                    // no more CTAs than slices of 4 ids per thread
+    while (C > 1 && (C / 2) * 4 * 512 >= n) C /= 2;                   // no more CTAs than slices of 4 ids per thread
     for (;; C *= 2) {
-        for (int ept = 4; ept <= 16; ept *= 2) {
-            if ((long long)C * ept * CT < n) continue;
-            if (ept == 16 && C < MAXC) break;                          // rather a larger cluster than 16 ids per thread
-            *C_out = C; *ept_out = ept;
-            return true;
+        for (int ept = 4; ept <= 8; ept *= 2)
+            if ((long long)C * ept * 512 >= n) { *C_out = C; *ept_out = ept; *ct_out = 512; return true; }
+        // long rows: rather a larger cluster than more ids per thread; at the largest cluster, 1024 threads
+        if (C >= MAXC) {
+            if ((long long)C * 8 * 1024 >= n) { *C_out = C; *ept_out = 8; *ct_out = 1024; return true; }
+            return false;
         }
-        if (C >= MAXC) return false;
     }
 }
 
@@ -729,10 +833,10 @@ bool choose_cluster(int n, int rows, int sm_count, int *C_out, int *ept_out)
 
 bool verify_cluster_supported(const VerifyParams &p)
 {
-    if (p.top_p24 != 0u || p.mode == SCD_MODE_SCD_GS) return false;   // nucleus and Gumbel race: the one-CTA kernel
-    if (p.L > CT) return false;
-    int C, ept;
-    return choose_cluster(p.allowed_hi - p.allowed_lo, p.L * p.B, 148, &C, &ept);
+    if (p.mode == SCD_MODE_SCD_GS) return false;                      // the Gumbel race: the one-CTA kernel
+    if (p.L > 512) return false;
+    int C, ept, ct;
+    return choose_cluster(p.allowed_hi - p.allowed_lo, p.L * p.B, 148, &C, &ept, &ct);
 }
 
 int launch_verify_cluster(const VerifyParams &p, cudaStream_t stream)
@@ -749,12 +853,12 @@ int launch_verify_cluster(const VerifyParams &p, cudaStream_t stream)
     });
     if (rc != SCD_OK) return rc;
     if (dev >= 0 && dev < DeviceOnce::kSlots) sms = sm_count[dev];
-    int C = 1, ept = 4;
-    SCD_REQUIRE(choose_cluster(p.allowed_hi - p.allowed_lo, p.L * p.B, sms, &C, &ept), SCD_ERR_SHAPE,
+    int C = 1, ept = 4, ct = 512;
+    SCD_REQUIRE(choose_cluster(p.allowed_hi - p.allowed_lo, p.L * p.B, sms, &C, &ept, &ct), SCD_ERR_SHAPE,
                 "verify: rows of %d ids do not fit a cluster", p.allowed_hi - p.allowed_lo);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(p.L * C), (unsigned)p.B, 1);
-    cfg.blockDim = dim3(CT, 1, 1);
+    cfg.blockDim = dim3((unsigned)ct, 1, 1);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
@@ -766,9 +870,9 @@ int launch_verify_cluster(const VerifyParams &p, cudaStream_t stream)
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    if (ept == 4) SCD_CUDA_TRY(cudaLaunchKernelEx(&cfg, verify_cluster_kernel<4>, p, C));
-    else if (ept == 8) SCD_CUDA_TRY(cudaLaunchKernelEx(&cfg, verify_cluster_kernel<8>, p, C));
-    else SCD_CUDA_TRY(cudaLaunchKernelEx(&cfg, verify_cluster_kernel<16>, p, C));
+    if (ct == 1024) SCD_CUDA_TRY(cudaLaunchKernelEx(&cfg, verify_cluster_kernel<8, 1024>, p, C));
+    else if (ept == 4) SCD_CUDA_TRY(cudaLaunchKernelEx(&cfg, verify_cluster_kernel<4, 512>, p, C));
+    else SCD_CUDA_TRY(cudaLaunchKernelEx(&cfg, verify_cluster_kernel<8, 512>, p, C));
     return SCD_OK;
 }
 
