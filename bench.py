@@ -29,11 +29,12 @@ UNIT = "tokens/s"
 
 # Typed-in constants (NOT measured by a run of this file; each is labelled as such in the JSON line).
 # DRAM traffic of gemm_ws_kernel relative to its algorithmic (weight) bytes, from the ncu capture
-# summarised in profiles/gemm_ws_kernel_qkv_shape.md (dram__bytes_read.sum + dram__bytes_write.sum over
-# the weight bytes of that launch). Traffic grows in proportion to the weight bytes (every weight is read
-# once), so the ratio is applied to the average launch. None = the kernel changed since the capture.
-GEMM_TRAFFIC_RATIO = None
-GEMM_TRAFFIC_SOURCE = "profiles/gemm_ws_kernel_qkv_shape.md (ncu capture; typed in, not measured by this run)"
+# summarised in profiles/gemm_ws_kernel_session_layer.md (dram__bytes_read.sum + dram__bytes_write.sum of
+# the four GEMMs of a layer over their weight bytes: 419.9 MB for 404.75 MB). Traffic grows in proportion
+# to the weight bytes (every weight is read once), so the ratio is applied to the average launch.
+# None = the kernel changed since the capture.
+GEMM_TRAFFIC_RATIO = 1.037
+GEMM_TRAFFIC_SOURCE = "profiles/gemm_ws_kernel_session_layer.md (ncu capture; typed in, not measured by this run)"
 
 # Tokens committed per forward on each workload, as measured by earlier runs of the CUDA arm (the oracle
 # commits the same tokens: parity). Used only by the reference arm, which cannot afford whole generations,
@@ -115,6 +116,8 @@ def config_of(args, shape):
             "prompt_len": shape["prompt_len"], "n_gen": shape["n_gen"], "top_k": shape["top_k"],
             "cfg_lambda": shape["cfg_lambda"], "coupling": args.coupling,
             "autotune": bool(getattr(args, "autotune", False)),
+            "layers": shape["n_layers"],
+            "truncated_for_profiling": bool(getattr(args, "layers", 0)),
             "l2": "inputs larger than L2 (weights streamed once per step)",
             "replicas": "one independent decode batch per GPU"}
 
@@ -563,9 +566,14 @@ def main():
     ap.add_argument("--no-contexts", action="store_true", help="skip the start / mid / end measurements")
     ap.add_argument("--context-steps", type=int, default=24, help="iterations timed at each of start / mid / end")
     ap.add_argument("--window", type=int, default=0, help="Jacobi window L (0 = the workload's)")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="profiling only: truncate the decoder to this many layers (a small model for ncu captures; "
+                         "the line is marked and is not a benchmark of the workload)")
     args = ap.parse_args()
     from paper_2510_24211_b200 import synth
     shape = dict(synth.WORKLOADS[args.workload])
+    if args.layers > 0:
+        shape["n_layers"] = min(shape["n_layers"], args.layers)
     if args.impl == "reference":
         # the oracle's steps are tens of seconds each: bound the run
         args.steps_ref = max(1, min(args.steps, 3))
