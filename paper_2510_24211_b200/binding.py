@@ -23,7 +23,7 @@ EXPORTS = (
     "scd_session_free", "scd_prefill", "scd_step", "scd_step_result", "scd_generate",
     "scd_read_tokens", "scd_verify_workspace_bytes", "scd_verify", "scd_forward_window",
     "scd_noise_u24", "scd_gemm_workspace_bytes", "scd_gemm_bf16", "scd_debug_read", "scd_model_gemm_tune", "scd_gemm_bf16_shaped", "scd_selftest_device_once",
-    "scd_step_profile", "scd_step_timeline", "scd_autotune", "scd_kernel_launches", "scd_verify_noalloc", "scd_verify_noalloc_max_bytes",
+    "scd_step_profile", "scd_step_timeline", "scd_session_attention_min_ctx", "scd_autotune", "scd_kernel_launches", "scd_verify_noalloc", "scd_verify_noalloc_max_bytes",
 )
 
 PROF_CLASSES = ("embed", "rmsnorm", "gemm_qkv", "rope_kv", "attention", "gemm_o", "gemm_gate_up",
@@ -127,6 +127,8 @@ def _declare(l):
     l.scd_autotune.restype = C.c_int
     l.scd_step_timeline.argtypes = [vp, vp, vp, vp]
     l.scd_step_timeline.restype = C.c_int
+    l.scd_session_attention_min_ctx.argtypes = [vp, C.c_int64]
+    l.scd_session_attention_min_ctx.restype = C.c_int
     l.scd_kernel_launches.argtypes = []
     l.scd_kernel_launches.restype = C.c_int64
     l.scd_gemm_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
@@ -354,6 +356,9 @@ class Session:
         out = np.zeros(4, dtype=np.int32)
         _check(lib().scd_autotune(self.handle, out.ctypes.data_as(C.c_void_p), _stream(stream)))
         return out
+
+    def scd_session_attention_min_ctx(self, min_ctx):
+        _check(lib().scd_session_attention_min_ctx(self.handle, int(min_ctx)))
 
     def scd_step_timeline(self, ms=None, launches=None, stream=None):
         """One iteration timed by device time stamps inside the kernels (no events between them)."""

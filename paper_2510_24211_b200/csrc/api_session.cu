@@ -108,8 +108,8 @@ void drop_step_graph(scd_session *s)
 int launch_step(scd_session *s, cudaStream_t st)
 {
     // the captured launches carry the attention variant: capture again when it changes (once per generation)
-    const bool wide = s->attn_plan && attention_tc_wide(s, s->L);
-    if (wide != s->att_wide) { s->att_wide = wide; drop_step_graph(s); }
+    const int variant = s->attn_plan ? attention_tc_variant(s, s->L) : 0;
+    if (variant != s->att_variant) { s->att_variant = variant; drop_step_graph(s); }
     struct Advance { scd_session *s; ~Advance() { s->ctx_floor += 1; } } advance{s};   // every iteration commits >= 1 token
     if (s->step_graph_off) return enqueue_step(s, st);
     if (!s->step_graph) {
@@ -249,6 +249,7 @@ int scd_session_create(scd_model_t *m, const scd_decode_config_t *cfg, scd_sessi
     s->Q = s->B * s->S;
     s->L = cfg->mode == SCD_MODE_AR ? 1 : cfg->window_L;
     s->cfg.window_L = s->L;
+    s->att_t5_min_ctx = 512;
     // rows one forward may carry per stream-sequence: the window, or a prefill chunk
     s->chunk = std::max(s->L, std::max(1, std::min(128, 256 / s->Q)));
     s->rows_cap = s->Q * s->chunk;
@@ -380,7 +381,7 @@ int scd_prefill(scd_session_t *s, const int32_t *prompt_ids, int32_t P, int32_t 
     rc = check_device_health(s, st);
     if (rc != SCD_OK) return rc;
     s->ctx_floor = (long long)P - 1;                   // kv_len after the prefill
-    s->att_wide = false;
+    s->att_variant = 0;
     s->prefilled = true;
     return SCD_OK;
 }
@@ -390,6 +391,13 @@ int scd_step(scd_session_t *s, void *stream)
     SCD_REQUIRE(s, SCD_ERR_ARG, "scd_step: NULL session");
     SCD_REQUIRE(s->prefilled, SCD_ERR_STATE, "scd_step before scd_prefill");
     return launch_step(s, (cudaStream_t)stream);
+}
+
+int scd_session_attention_min_ctx(scd_session_t *s, int64_t min_ctx)
+{
+    SCD_REQUIRE(s, SCD_ERR_ARG, "scd_session_attention_min_ctx: NULL session");
+    s->att_t5_min_ctx = (long long)min_ctx;
+    return SCD_OK;
 }
 
 int scd_step_profile(scd_session_t *s, float *ms_by_class, int32_t *launches_by_class, void *stream)

@@ -48,7 +48,8 @@ struct scd_session {
     int ss_parts_cap;
     float *logits;            // [rows_cap_logits][V]
     long long ctx_floor;      // host-side floor of the committed context of every live sequence (P - 1 + iterations)
-    bool att_wide;            // attention variant the captured iteration was built with
+    int att_variant;          // attention variant the captured iteration was built with
+    long long att_t5_min_ctx; // known context from which the tcgen05 attention kernel is used (< 0: never)
     void *stamps;             // device time stamps of scd_step_timeline (allocated on first use)
     void *gemm_ws;            // device error word of the tcgen05 GEMM
     size_t gemm_ws_bytes;

@@ -95,11 +95,13 @@ MID_BF16_D128_GQA = dict(n_layers=2, d_model=256, n_heads=2, n_kv_heads=1, head_
     (MID_BF16_D128_GQA, 128, 1500, 16),  # the same with head_dim 128 and a window CTA without context tiles
     (MID_BF16_D128_GQA, 64, 1100, 1),  # single row, long context
 ])
-def test_forward_tensor_core_attention(shape, page, P, M):
+@pytest.mark.parametrize("kernel", ["mma_sync", "tcgen05"])
+def test_forward_tensor_core_attention(shape, page, P, M, kernel):
     gm, om = _models(shape, max_seq=P + 2 * M + 70, seed=9, std=0.08, page=page)
     rng = np.random.default_rng(P)
     prompt = rng.integers(0, shape["vocab_in"], size=(1, P)).astype(np.int32)
     sess = scd.Session(gm, scd.decode_config(batch=1, window_L=M, allowed_hi=shape["vocab_out"]))
+    sess.scd_session_attention_min_ctx(0 if kernel == "tcgen05" else -1)   # every context length through each kernel
     sess.scd_prefill(prompt, n_new=M + 40)
     om.forward(prompt[0, :-1], 0)
     ids = np.concatenate([prompt[0, -1:], rng.integers(0, shape["vocab_in"], size=M - 1)]).astype(np.int32)
@@ -115,14 +117,17 @@ def test_forward_tensor_core_attention(shape, page, P, M):
         assert _rel(logits2[0].cpu().numpy(), ref2) <= 3e-2
 
 
-def test_step_replay_bf16_tensor_core_attention_cfg_batch():
-    # CFG pair of streams x 2 sequences through the tensor-core attention and the cluster GEMMs
+@pytest.mark.parametrize("att_min_ctx", [-1, 0])
+def test_step_replay_bf16_tensor_core_attention_cfg_batch(att_min_ctx):
+    # CFG pair of streams x 2 sequences through the tensor-core attention (the mma.sync kernel, then the
+    # tcgen05 kernel, inside the captured iteration) and the cluster GEMMs
     _replay_case(MID_BF16_D64, oracle.MODE_SCD_MC, B=2, L=16, P=70, n_new=60, top_k=40, lam=2.0, seed=8,
-                 page=64)
+                 page=64, att_min_ctx=att_min_ctx)
 
 
 def _replay_case(shape, mode, B, L, P, n_new, top_k, lam=0.0, temperature=1.0, seed=0, lo=0, hi=None,
-                 row_period=0, eol_id=0, std=0.3, page=16, alpha=1.0, top_p=0.0, autotune=False, gm=None):
+                 row_period=0, eol_id=0, std=0.3, page=16, alpha=1.0, top_p=0.0, autotune=False, gm=None,
+                 att_min_ctx=None):
     """Run the GPU session step by step, then replay its logits through the oracle's loop."""
     hi = shape["vocab_out"] if hi is None else hi
     S = 2 if lam != 0.0 else 1
@@ -136,6 +141,8 @@ def _replay_case(shape, mode, B, L, P, n_new, top_k, lam=0.0, temperature=1.0, s
                             cfg_lambda=lam, seed=seed, allowed_lo=lo, allowed_hi=hi,
                             row_period=row_period, eol_id=eol_id, alpha=alpha, top_p=top_p)
     sess = scd.Session(gm, cfg)
+    if att_min_ctx is not None:
+        sess.scd_session_attention_min_ctx(att_min_ctx)
     sess.scd_prefill(prompts, n_new=n_new)
     if autotune:
         before = [x.copy() for x in sess.scd_step_result()] + [sess.scd_debug_read("drafts").copy()]
