@@ -297,6 +297,8 @@ def run_scd(args, shape):
     coupling = {"scd_mc": scd.SCD_MODE_SCD_MC, "scd_gs": scd.SCD_MODE_SCD_GS, "sjd": scd.SCD_MODE_SJD,
                 "alpha": scd.SCD_MODE_ALPHA}[args.coupling]
     sess = scd.Session(model, cfg_of(coupling))
+    if args.att_min_ctx is not None:
+        sess.scd_session_attention_min_ctx(args.att_min_ctx)
     tuned = None
     stream = torch.cuda.current_stream()
     peaks = measured_peaks()
@@ -566,6 +568,9 @@ def main():
     ap.add_argument("--no-contexts", action="store_true", help="skip the start / mid / end measurements")
     ap.add_argument("--context-steps", type=int, default=24, help="iterations timed at each of start / mid / end")
     ap.add_argument("--window", type=int, default=0, help="Jacobi window L (0 = the workload's)")
+    ap.add_argument("--att-min-ctx", type=int, default=None,
+                    help="tuning: committed context from which the tcgen05 attention kernel is used (default: the library's; "
+                         "0 = always, -1 = never)")
     ap.add_argument("--layers", type=int, default=0,
                     help="profiling only: truncate the decoder to this many layers (a small model for ncu captures; "
                          "the line is marked and is not a benchmark of the workload)")

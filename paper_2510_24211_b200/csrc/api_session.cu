@@ -168,9 +168,11 @@ int check_device_health(scd_session *s, cudaStream_t st)
     if (rc != SCD_OK) return rc;
     static const char *const who[] = {"", "GEMM: producer waiting for a free ring slot", "GEMM: MMA issuer waiting for operands",
                                       "GEMM: epilogue waiting for the accumulator", "attention: waiting for a free ring slot",
-                                      "attention: waiting for a K/V tile", "attention: shared memory base not 1024-byte aligned"};
+                                      "attention: waiting for a K/V tile", "attention: shared memory base not 1024-byte aligned",
+                                      "attention: softmax waiting for the scores", "attention: waiting for the probabilities",
+                                      "attention: waiting for the product P V", "attention: waiting for a free score buffer"};
     SCD_REQUIRE(word == 0, SCD_ERR_TIMEOUT, "a bounded device-side wait gave up (%s, code %d); prefill the session again",
-                word > 0 && word < 7 ? who[word] : "unknown", word);
+                word > 0 && word < 11 ? who[word] : "unknown", word);
     return SCD_OK;
 }
 

@@ -685,12 +685,6 @@ __device__ __forceinline__ uint64_t t5_desc_mn(uint32_t smem_addr, uint32_t lbo_
     return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) | (64ull << 32) |
            (1ull << 46) | (2ull << 61);
 }
-__device__ __forceinline__ void t5_mma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc)
-{
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
-}
 // A bounded wait that gives up early when another thread of the CTA already has (`failed`).
 __device__ __forceinline__ bool t5_wait(uint64_t *bar, unsigned parity, volatile int *failed)
 {
@@ -706,7 +700,8 @@ __device__ __forceinline__ bool t5_wait(uint64_t *bar, unsigned parity, volatile
     }
     return false;
 }
-// the same with the A operand in tensor memory (lane = row, 32-bit column c = elements 2c, 2c + 1 of the row)
+// D (+)= A B with the A operand in tensor memory (lane = row, 32-bit column c = elements 2c, 2c + 1 of the row)
+// and B in shared memory
 __device__ __forceinline__ void t5_mma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t db, uint32_t idesc, uint32_t acc)
 {
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
@@ -745,10 +740,6 @@ __device__ __forceinline__ float t5_ex2(float x)
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
-}
-__device__ __forceinline__ void t5_st4(uint32_t taddr, uint4 v)
-{
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 template <int N>
 __device__ __forceinline__ void t5_st_u32(uint32_t taddr, const uint32_t *v)   // N = 8, 16, 32 consecutive columns
@@ -1013,7 +1004,7 @@ __global__ void __launch_bounds__(T5_THREADS, 1) attention_t5_kernel(const __gri
     // the k steps of one tile differ only in the start address field (bits 0-13, in 16-byte units; shared memory
     // ends far below 2^18 bytes, so adding there never carries out).
     auto mma_s = [&](int t, uint32_t kaddr) {
-        if (t >= 2) wait_on(&bar_sc[t & 1], (unsigned)((t - 2) >> 1) & 1u, 3);
+        if (t >= 2) wait_on(&bar_sc[t & 1], (unsigned)((t - 2) >> 1) & 1u, 10);
         const uint32_t d = tmem_s + (uint32_t)(t & 1) * 64u;
         const uint64_t dk = t5_desc_k(kaddr);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -1210,41 +1201,58 @@ __global__ void __launch_bounds__(T5_THREADS, 1) attention_t5_kernel(const __gri
     if (C > 1) {
         __syncwarp();
         cluster_sync_all();
-        {
-            const int r_lo = (int)(((long long)rank * rows) / C), r_hi = (int)(((long long)(rank + 1) * rows) / C);
-            const int nr = r_hi - r_lo;
-            const uint32_t o_addr = smem_u32(o_st), m_addr = smem_u32(m2_st), l_addr = smem_u32(l2_st);
-            for (int e = tid; e < nr * (DH / 4); e += T5_THREADS) {
-                const int rl = e / (DH / 4), rr = r_lo + rl, col = (e % (DH / 4)) * 4;
-                float4 part[8];
-                float mp[8], lp[8];
+        const int r_lo = (int)(((long long)rank * rows) / C), r_hi = (int)(((long long)(rank + 1) * rows) / C);
+        const int nr = r_hi - r_lo;                                // rows this CTA merges and writes
+        const uint32_t o_addr = smem_u32(o_st), m_addr = smem_u32(m2_st), l_addr = smem_u32(l2_st);
+        // every peer's maximum and sum of these rows: one (row, peer) per thread, into local arrays
+        float *pm_st = l2_st + 128, *pl_st = pm_st + 136;
+        for (int j = tid; j < nr * C; j += T5_THREADS) {
+            const int rl = j / C, peer = j - rl * C;
+            pm_st[j] = ld_cluster_f32(map_peer(m_addr + (uint32_t)(r_lo + rl) * 4u, (uint32_t)peer));
+            pl_st[j] = ld_cluster_f32(map_peer(l_addr + (uint32_t)(r_lo + rl) * 4u, (uint32_t)peer));
+        }
+        // four dims of a row per item, two items per thread at a time: the remote loads of both are in flight
+        // together, and with the scalar loads above
+        const int n_items = nr * (DH / 4);
+        const int n_rounds = (n_items + 2 * T5_THREADS - 1) / (2 * T5_THREADS);   // (the same in every thread)
+        for (int round = 0; round < n_rounds; ++round) {
+            const int e0 = tid + round * 2 * T5_THREADS;
+            float4 part[2][8];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int e = e0 + u * T5_THREADS;
+                const int rr = r_lo + e / (DH / 4), col = (e % (DH / 4)) * 4;
 #pragma unroll
                 for (int peer = 0; peer < 8; ++peer) {
-                    part[peer] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    mp[peer] = -INFINITY;
-                    lp[peer] = 0.f;
-                    if (peer < C) {
-                        part[peer] = ld_cluster_f32x4(map_peer(o_addr + (uint32_t)(rr * OROW + col) * 4u, (uint32_t)peer));
-                        mp[peer] = ld_cluster_f32(map_peer(m_addr + rr * 4u, (uint32_t)peer));
-                        lp[peer] = ld_cluster_f32(map_peer(l_addr + rr * 4u, (uint32_t)peer));
-                    }
+                    part[u][peer] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (peer < C && e < n_items)
+                        part[u][peer] = ld_cluster_f32x4(map_peer(o_addr + (uint32_t)(rr * OROW + col) * 4u, (uint32_t)peer));
                 }
-                float M = -INFINITY;
+            }
+            if (round == 0) __syncthreads();                      // the local arrays are complete
 #pragma unroll
-                for (int peer = 0; peer < 8; ++peer) M = fmaxf(M, mp[peer]);
-                float L = 0.f;
+            for (int u = 0; u < 2; ++u) {
+                const int e = e0 + u * T5_THREADS;
+                if (e >= n_items) break;
+                const int rl = e / (DH / 4), rr = r_lo + rl, col = (e % (DH / 4)) * 4;
+                float wp[8], M = -INFINITY, L = 0.f;
 #pragma unroll
                 for (int peer = 0; peer < 8; ++peer) {
-                    mp[peer] = mp[peer] == -INFINITY ? 0.f : exp2f(mp[peer] - M);
-                    L += mp[peer] * lp[peer];
+                    wp[peer] = peer < C ? pm_st[rl * C + peer] : -INFINITY;
+                    M = fmaxf(M, wp[peer]);
+                }
+#pragma unroll
+                for (int peer = 0; peer < 8; ++peer) {
+                    wp[peer] = wp[peer] == -INFINITY ? 0.f : exp2f(wp[peer] - M);
+                    if (peer < C) L += wp[peer] * pl_st[rl * C + peer];
                 }
                 const float inv = L > 0.f ? 1.0f / L : 0.f;
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                 for (int peer = 0; peer < 8; ++peer) {
-                    const float wp = mp[peer] * inv;
-                    acc.x += wp * part[peer].x; acc.y += wp * part[peer].y;
-                    acc.z += wp * part[peer].z; acc.w += wp * part[peer].w;
+                    const float w8 = wp[peer] * inv;
+                    acc.x += w8 * part[u][peer].x; acc.y += w8 * part[u][peer].y;
+                    acc.z += w8 * part[u][peer].z; acc.w += w8 * part[u][peer].w;
                 }
                 const int i = rr % Mq, gq = rr / Mq;
                 __nv_bfloat16 *dst = p.out + ((size_t)q * Mq + i) * ostride + (size_t)(kvh * p.n_rep + gq) * DH + col;
@@ -1272,6 +1280,7 @@ __global__ void __launch_bounds__(T5_THREADS, 1) attention_t5_kernel(const __gri
 struct AttnPlan {
     CUtensorMap kv_map;
     int sm_count;
+    int t5_rows, t5_C;        // tcgen05 kernel: cluster size found for windows of t5_rows query rows (0: not looked for yet)
 };
 
 }  // namespace
@@ -1323,93 +1332,134 @@ static int attention_clusters(const scd_session *s, const AttnPlan *plan)
     return C;
 }
 
-// The tcgen05 kernel runs one CTA per SM: its clusters must fit one wave of sm_count CTAs.
-static int attention_clusters_t5(const scd_session *s, const AttnPlan *plan)
+
+using T5Kernel = void (*)(const AttnParams);
+constexpr size_t T5_SMEM = 227 * 1024 - 8192;   // all of an SM's shared memory but the kernel's static part (some 5 KB)
+
+static T5Kernel t5_kernel(int dh, int rows, int *G_out)
 {
-    const scd_model_config_t &c = s->model->cfg;
-    const int units = s->Q * c.n_kv_heads;
-    const int c_cap = std::max(1, std::min(8, plan->sm_count / std::max(1, units)));
-    int C = 1;
-    while (C * 2 <= c_cap) C *= 2;
-    return C;
+    const int G = rows > 64 ? 1 : rows > 32 ? 2 : 4;              // column groups: 128 / G query rows per CTA
+    *G_out = G;
+    return dh == 128 ? (G == 1 ? attention_t5_kernel<128, 1> : G == 2 ? attention_t5_kernel<128, 2> : attention_t5_kernel<128, 4>)
+                     : (G == 1 ? attention_t5_kernel<64, 1> : G == 2 ? attention_t5_kernel<64, 2> : attention_t5_kernel<64, 4>);
 }
 
-// 0: one warp per query tile; 1: two warps per query tile; 2: the tcgen05 kernel (decoding steps only:
-// at most 128 query rows per KV head, the units fit one wave, and every CTA has a few key tiles to work on)
+// The largest cluster the tcgen05 kernel may use for windows of `rows` query rows: one CTA per SM and one wave,
+// i.e. the device must hold one cluster per (sequence, KV head) at the same time. Any size up to 8 (the kernel
+// splits tiles and rows evenly). The answer depends on how the SMs are grouped, so the runtime is asked - once.
+static int t5_max_cluster(const scd_session *s, AttnPlan *plan, int rows)
+{
+    if (plan->t5_rows == rows) return plan->t5_C;
+    const scd_model_config_t &c = s->model->cfg;
+    const int units = s->Q * c.n_kv_heads;
+    static DeviceOnce once;
+    int dev = 0;
+    if (current_device(&dev) != SCD_OK) return 0;
+    const int rc = once.run(dev, [&]() -> int {
+        SCD_CUDA_TRY(cudaFuncSetAttribute(attention_t5_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)T5_SMEM));
+        SCD_CUDA_TRY(cudaFuncSetAttribute(attention_t5_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)T5_SMEM));
+        SCD_CUDA_TRY(cudaFuncSetAttribute(attention_t5_kernel<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)T5_SMEM));
+        SCD_CUDA_TRY(cudaFuncSetAttribute(attention_t5_kernel<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)T5_SMEM));
+        SCD_CUDA_TRY(cudaFuncSetAttribute(attention_t5_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)T5_SMEM));
+        SCD_CUDA_TRY(cudaFuncSetAttribute(attention_t5_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)T5_SMEM));
+        return SCD_OK;
+    });
+    if (rc != SCD_OK) return 0;
+    int G = 1;
+    const T5Kernel fn = t5_kernel(c.head_dim, rows, &G);
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cfg.blockDim = dim3(T5_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = T5_SMEM;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 1;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int best = 1;
+    for (int C = std::min(8, plan->sm_count / std::max(1, units)); C >= 2; --C) {
+        cfg.gridDim = dim3((unsigned)(units * C), 1, 1);
+        attr.val.clusterDim.x = (unsigned)C;
+        int fit = 0;
+        if (cudaOccupancyMaxActiveClusters(&fit, fn, &cfg) == cudaSuccess && fit >= units) { best = C; break; }
+        cudaGetLastError();
+    }
+    plan->t5_rows = rows;
+    plan->t5_C = best;
+    return best;
+}
+
+// Cluster size for a context of at least `tiles` key tiles: a CTA works about 0.85 us per tile (its share of the
+// context plus one for the window), and a cluster of more than one pays about 3.5 us for the exchange and the
+// merge of its parts.
+static int t5_pick_cluster(int c_max, long long tiles)
+{
+    int best = 1;
+    double best_us = 1e30;
+    for (int C = 1; C <= c_max; ++C) {
+        const double us = 0.85 * (double)((tiles + C - 1) / C + 1) + (C > 1 ? 3.5 : 0.0);
+        if (us < best_us - 1e-9) { best_us = us; best = C; }
+    }
+    return best;
+}
+
+// Low 4 bits: 0 = one warp per query tile; 1 = two warps per query tile; 2 = the tcgen05 kernel (decoding steps only:
+// at most 128 query rows per KV head, the units fit one wave), with its cluster size in the bits above. The choice
+// follows the host's floor of the context length; a captured iteration is built for one value of it.
 int attention_tc_variant(const scd_session *s, int Mq)
 {
     const scd_model_config_t &c = s->model->cfg;
-    const AttnPlan *plan = (const AttnPlan *)s->attn_plan;
+    AttnPlan *plan = (AttnPlan *)s->attn_plan;
     if (!plan) return 0;
     const int rows = Mq * (c.n_heads / c.n_kv_heads);
     const long long tiles = (std::max(0ll, s->ctx_floor) + TK - 1) / TK;
     if (rows <= 128 && s->Q * c.n_kv_heads <= plan->sm_count && (c.max_seq + TK - 1) / TK <= T5_MAX_TILES && s->att_t5_min_ctx >= 0 &&
-        s->ctx_floor >= s->att_t5_min_ctx)
-        return 2;
+        s->ctx_floor >= s->att_t5_min_ctx) {
+        const int c_max = t5_max_cluster(s, plan, rows);
+        if (c_max >= 1) return 2 | (t5_pick_cluster(c_max, tiles) << 4);
+    }
     const int n_mtiles = (rows + 15) / 16;
     if (n_mtiles > 2) return 0;
     const int C = attention_clusters(s, plan);
     return (tiles + 3 + C - 1) / C >= 4 ? 1 : 0;
 }
 
-static int attention_t5(scd_session *s, AttnParams &p, cudaStream_t st)
+static int attention_t5(scd_session *s, AttnParams &p, int C, cudaStream_t st)
 {
     const scd_model_config_t &c = s->model->cfg;
-    AttnPlan *plan = (AttnPlan *)s->attn_plan;
     const int dh = c.head_dim, units = s->Q * c.n_kv_heads;
-    p.C = attention_clusters_t5(s, plan);
     const int rows = p.Mq * p.n_rep;
-    const int G = rows > 64 ? 1 : rows > 32 ? 2 : 4;              // column groups: 128 / G query rows per CTA
+    int G = 1;
+    const T5Kernel fn = t5_kernel(dh, rows, &G);
     const size_t tile_bytes = (size_t)TK * dh * 2;                // one K or V slot
-    const size_t merge_bytes = (size_t)128 * (dh + 4 + 4) * sizeof(float);
-    // All of the SM's shared memory but the kernel's static part: no CTA of another kernel fits beside this
-    // one, so the tensor memory - all 512 columns - is never contended for (see the kernel's header).
-    const size_t lim = 227 * 1024 - 8192;
-    // the rotated queries on their way to tensor memory, then the window's K and V tiles
+    const size_t merge_bytes = (size_t)128 * (dh + 4 + 8) * sizeof(float);
+    // All the shared memory a CTA can have: no CTA of another kernel fits beside this one, so the tensor
+    // memory - all 512 columns - is never contended for (see the kernel's header).
+    // Behind the rings: the rotated queries on their way to tensor memory, then the window's K and V tiles.
     const size_t q_stage = std::max((size_t)2 * (128 / G) * (dh * 2 + 16), (size_t)2 * ((p.Mq + TK - 1) / TK) * tile_bytes);
-    const int slots = (int)std::min<size_t>(2 * MAX_ATT_STAGES, (lim - q_stage) / tile_bytes);
+    const int slots = (int)std::min<size_t>(2 * MAX_ATT_STAGES, (T5_SMEM - q_stage) / tile_bytes);
     SCD_REQUIRE(slots >= 4 && (size_t)slots * tile_bytes >= merge_bytes, SCD_ERR_SHAPE, "attention: shared memory does not fit");
     p.stages = slots / 2;                                         // K ring
     p.stages_v = slots - slots / 2;                               // V ring: a V slot is held longer
-    const size_t smem = lim;
-    static DeviceOnce once;
-    int dev = 0;
-    int rc = current_device(&dev);
-    if (rc != SCD_OK) return rc;
-    rc = once.run(dev, [&]() -> int {
-        SCD_CUDA_TRY(cudaFuncSetAttribute(attention_t5_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lim));
-        SCD_CUDA_TRY(cudaFuncSetAttribute(attention_t5_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lim));
-        SCD_CUDA_TRY(cudaFuncSetAttribute(attention_t5_kernel<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lim));
-        SCD_CUDA_TRY(cudaFuncSetAttribute(attention_t5_kernel<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lim));
-        SCD_CUDA_TRY(cudaFuncSetAttribute(attention_t5_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lim));
-        SCD_CUDA_TRY(cudaFuncSetAttribute(attention_t5_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lim));
-        return SCD_OK;
-    });
-    if (rc != SCD_OK) return rc;
+    p.C = C;
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof(cfg));
-    cfg.gridDim = dim3((unsigned)(units * p.C), 1, 1);
+    cfg.gridDim = dim3((unsigned)(units * C), 1, 1);
     cfg.blockDim = dim3(T5_THREADS, 1, 1);
-    cfg.dynamicSmemBytes = smem;
+    cfg.dynamicSmemBytes = T5_SMEM;
     cfg.stream = st;
     cudaLaunchAttribute attrs[2];
-    attrs[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attrs[0].val.programmaticStreamSerializationAllowed = 1;
-    attrs[1].id = cudaLaunchAttributeClusterDimension;
-    attrs[1].val.clusterDim.x = (unsigned)p.C;
-    attrs[1].val.clusterDim.y = 1;
-    attrs[1].val.clusterDim.z = 1;
+    attrs[0].id = cudaLaunchAttributeClusterDimension;
+    attrs[0].val.clusterDim.x = (unsigned)C;
+    attrs[0].val.clusterDim.y = 1;
+    attrs[0].val.clusterDim.z = 1;
+    attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attrs[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attrs;
     cfg.numAttrs = 2;
-    if (dh == 128) {
-        if (G == 1) SCD_CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_t5_kernel<128, 1>, p));
-        else if (G == 2) SCD_CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_t5_kernel<128, 2>, p));
-        else SCD_CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_t5_kernel<128, 4>, p));
-    } else {
-        if (G == 1) SCD_CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_t5_kernel<64, 1>, p));
-        else if (G == 2) SCD_CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_t5_kernel<64, 2>, p));
-        else SCD_CUDA_TRY(cudaLaunchKernelEx(&cfg, attention_t5_kernel<64, 4>, p));
-    }
+    SCD_CUDA_TRY(cudaLaunchKernelEx(&cfg, fn, p));
     count_launches(1);
     return SCD_OK;
 }
@@ -1441,7 +1491,7 @@ int attention_tc(scd_session *s, int layer, int Mq, int pos_override, cudaStream
     p.n_mtiles = (Mq * p.n_rep + 15) / 16;
     p.qscale = 1.4426950408889634f / sqrtf((float)c.head_dim);
     const int variant = pos_override < 0 ? attention_tc_variant(s, Mq) : 0;
-    if (variant == 2) return attention_t5(s, p, st);
+    if ((variant & 15) == 2) return attention_t5(s, p, variant >> 4, st);
     const int units = s->Q * c.n_kv_heads;
     // split-KV over a cluster: up to two CTAs per SM over the whole grid, a power of two (measured:
     // clusters of 7 take 1.8 times as long as clusters of 4 on the same problem)
@@ -1485,7 +1535,7 @@ int attention_tc(scd_session *s, int layer, int Mq, int pos_override, cudaStream
         return SCD_OK;
     });
     if (rc != SCD_OK) return rc;
-    const bool wide = variant == 1;                               // two warps per query tile
+    const bool wide = (variant & 15) == 1;                        // two warps per query tile
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)(units * p.C), 1, 1);

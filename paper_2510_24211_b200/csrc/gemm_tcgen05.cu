@@ -494,13 +494,14 @@ __global__ void __launch_bounds__(GEMM_THREADS, 3) gemm_ws_kernel(const __grid_c
         };
         for (int i = 0; i < pre; ++i) load_x(i, i);
         int issued = pre;
-        for (int i = pre; i < nk; ++i) {
-            const int s = i % p.stages, round = i / p.stages;
+        // (slot and round as running counters: a division per K block is a long way for one lane)
+        for (int i = pre, s = pre == p.stages ? 0 : pre, round = pre == p.stages ? 1 : 0; i < nk; ++i) {
             if (!mbar_wait(&empty_bar[s], (round & 1) ^ 1)) { atomicExch(p.err, 1); abort_flag = 1; break; }
             mbar_expect_tx(&full_bar[s], load_bytes);
             load_w(i, s);
             load_x(i, s);
             issued = i + 1;
+            if (++s == p.stages) { s = 0; ++round; }
         }
         if (abort_flag) {
             // drain: give the copies already issued a bounded time to land before the CTA exits
@@ -512,20 +513,22 @@ __global__ void __launch_bounds__(GEMM_THREADS, 3) gemm_ws_kernel(const __grid_c
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(acc_cols >> 3) << 17) |
                                ((uint32_t)(TILE_N >> 4) << 24);
         bool ok = true;
-        for (int i = 0; i < nk && ok; ++i) {
-            const int s = i % p.stages, round = i / p.stages;
+        const bool second = p.x_planes == 2 && !fused2;
+        for (int i = 0, s = 0, round = 0; i < nk && ok; ++i) {
             ok = mbar_wait(&full_bar[s], round & 1);
             if (!ok) { atomicExch(p.err, 2); break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t sa = smem_u32(stage_base + (size_t)s * stage_bytes);
-            const uint32_t sb = sa + a_bytes;
+            // (the descriptors of the K steps differ in the start address field only: 16-byte units, no carry out of it)
+            const uint64_t da = umma_desc(sa), db = umma_desc(sa + a_bytes), db2 = umma_desc(sa + a_bytes + b_plane);
 #pragma unroll
             for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
-                const uint32_t koff = k * UMMA_K * 2;
-                umma_bf16(tmem_base, umma_desc(sa + koff), umma_desc(sb + koff), idesc, (i > 0 || k > 0) ? 1u : 0u);
-                if (p.x_planes == 2 && !fused2) umma_bf16(tmem_base, umma_desc(sa + koff), umma_desc(sb + b_plane + koff), idesc, 1u);
+                const uint32_t koff = (uint32_t)(k * UMMA_K * 2) >> 4;
+                umma_bf16(tmem_base, da + koff, db + koff, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                if (second) umma_bf16(tmem_base, da + koff, db2 + koff, idesc, 1u);
             }
             umma_commit(&empty_bar[s]);        // frees the slot once these MMAs have read it
+            if (++s == p.stages) { s = 0; ++round; }
         }
         umma_commit(&acc_bar);                 // accumulator complete (or abandoned)
     }

@@ -74,3 +74,4 @@ def test_calls_that_need_no_device():
     assert lib.scd_gemm_workspace_bytes(300, 4096, 4096) < 0     # more than 256 window rows
     with pytest.raises(scd.ScdError):
         scd._check(lib.scd_prefill(None, None, 1, 1, None))
+    assert lib.scd_session_attention_min_ctx(None, 0) < 0           # null session
