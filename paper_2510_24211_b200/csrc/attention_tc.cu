@@ -1201,58 +1201,41 @@ __global__ void __launch_bounds__(T5_THREADS, 1) attention_t5_kernel(const __gri
     if (C > 1) {
         __syncwarp();
         cluster_sync_all();
-        const int r_lo = (int)(((long long)rank * rows) / C), r_hi = (int)(((long long)(rank + 1) * rows) / C);
-        const int nr = r_hi - r_lo;                                // rows this CTA merges and writes
-        const uint32_t o_addr = smem_u32(o_st), m_addr = smem_u32(m2_st), l_addr = smem_u32(l2_st);
-        // every peer's maximum and sum of these rows: one (row, peer) per thread, into local arrays
-        float *pm_st = l2_st + 128, *pl_st = pm_st + 136;
-        for (int j = tid; j < nr * C; j += T5_THREADS) {
-            const int rl = j / C, peer = j - rl * C;
-            pm_st[j] = ld_cluster_f32(map_peer(m_addr + (uint32_t)(r_lo + rl) * 4u, (uint32_t)peer));
-            pl_st[j] = ld_cluster_f32(map_peer(l_addr + (uint32_t)(r_lo + rl) * 4u, (uint32_t)peer));
-        }
-        // four dims of a row per item, two items per thread at a time: the remote loads of both are in flight
-        // together, and with the scalar loads above
-        const int n_items = nr * (DH / 4);
-        const int n_rounds = (n_items + 2 * T5_THREADS - 1) / (2 * T5_THREADS);   // (the same in every thread)
-        for (int round = 0; round < n_rounds; ++round) {
-            const int e0 = tid + round * 2 * T5_THREADS;
-            float4 part[2][8];
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                const int e = e0 + u * T5_THREADS;
-                const int rr = r_lo + e / (DH / 4), col = (e % (DH / 4)) * 4;
-#pragma unroll
-                for (int peer = 0; peer < 8; ++peer) {
-                    part[u][peer] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (peer < C && e < n_items)
-                        part[u][peer] = ld_cluster_f32x4(map_peer(o_addr + (uint32_t)(rr * OROW + col) * 4u, (uint32_t)peer));
-                }
-            }
-            if (round == 0) __syncthreads();                      // the local arrays are complete
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                const int e = e0 + u * T5_THREADS;
-                if (e >= n_items) break;
+        {
+            const int r_lo = (int)(((long long)rank * rows) / C), r_hi = (int)(((long long)(rank + 1) * rows) / C);
+            const int nr = r_hi - r_lo;
+            const uint32_t o_addr = smem_u32(o_st), m_addr = smem_u32(m2_st), l_addr = smem_u32(l2_st);
+            for (int e = tid; e < nr * (DH / 4); e += T5_THREADS) {
                 const int rl = e / (DH / 4), rr = r_lo + rl, col = (e % (DH / 4)) * 4;
-                float wp[8], M = -INFINITY, L = 0.f;
+                float4 part[8];
+                float mp[8], lp[8];
 #pragma unroll
                 for (int peer = 0; peer < 8; ++peer) {
-                    wp[peer] = peer < C ? pm_st[rl * C + peer] : -INFINITY;
-                    M = fmaxf(M, wp[peer]);
+                    part[peer] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    mp[peer] = -INFINITY;
+                    lp[peer] = 0.f;
+                    if (peer < C) {
+                        part[peer] = ld_cluster_f32x4(map_peer(o_addr + (uint32_t)(rr * OROW + col) * 4u, (uint32_t)peer));
+                        mp[peer] = ld_cluster_f32(map_peer(m_addr + rr * 4u, (uint32_t)peer));
+                        lp[peer] = ld_cluster_f32(map_peer(l_addr + rr * 4u, (uint32_t)peer));
+                    }
                 }
+                float M = -INFINITY;
+#pragma unroll
+                for (int peer = 0; peer < 8; ++peer) M = fmaxf(M, mp[peer]);
+                float L = 0.f;
 #pragma unroll
                 for (int peer = 0; peer < 8; ++peer) {
-                    wp[peer] = wp[peer] == -INFINITY ? 0.f : exp2f(wp[peer] - M);
-                    if (peer < C) L += wp[peer] * pl_st[rl * C + peer];
+                    mp[peer] = mp[peer] == -INFINITY ? 0.f : exp2f(mp[peer] - M);
+                    L += mp[peer] * lp[peer];
                 }
                 const float inv = L > 0.f ? 1.0f / L : 0.f;
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                 for (int peer = 0; peer < 8; ++peer) {
-                    const float w8 = wp[peer] * inv;
-                    acc.x += w8 * part[u][peer].x; acc.y += w8 * part[u][peer].y;
-                    acc.z += w8 * part[u][peer].z; acc.w += w8 * part[u][peer].w;
+                    const float wp = mp[peer] * inv;
+                    acc.x += wp * part[peer].x; acc.y += wp * part[peer].y;
+                    acc.z += wp * part[peer].z; acc.w += wp * part[peer].w;
                 }
                 const int i = rr % Mq, gq = rr / Mq;
                 __nv_bfloat16 *dst = p.out + ((size_t)q * Mq + i) * ostride + (size_t)(kvh * p.n_rep + gq) * DH + col;
@@ -1391,20 +1374,6 @@ static int t5_max_cluster(const scd_session *s, AttnPlan *plan, int rows)
     return best;
 }
 
-// Cluster size for a context of at least `tiles` key tiles: a CTA works about 0.85 us per tile (its share of the
-// context plus one for the window), and a cluster of more than one pays about 3.5 us for the exchange and the
-// merge of its parts.
-static int t5_pick_cluster(int c_max, long long tiles)
-{
-    int best = 1;
-    double best_us = 1e30;
-    for (int C = 1; C <= c_max; ++C) {
-        const double us = 0.85 * (double)((tiles + C - 1) / C + 1) + (C > 1 ? 3.5 : 0.0);
-        if (us < best_us - 1e-9) { best_us = us; best = C; }
-    }
-    return best;
-}
-
 // Low 4 bits: 0 = one warp per query tile; 1 = two warps per query tile; 2 = the tcgen05 kernel (decoding steps only:
 // at most 128 query rows per KV head, the units fit one wave), with its cluster size in the bits above. The choice
 // follows the host's floor of the context length; a captured iteration is built for one value of it.
@@ -1418,7 +1387,10 @@ int attention_tc_variant(const scd_session *s, int Mq)
     if (rows <= 128 && s->Q * c.n_kv_heads <= plan->sm_count && (c.max_seq + TK - 1) / TK <= T5_MAX_TILES && s->att_t5_min_ctx >= 0 &&
         s->ctx_floor >= s->att_t5_min_ctx) {
         const int c_max = t5_max_cluster(s, plan, rows);
-        if (c_max >= 1) return 2 | (t5_pick_cluster(c_max, tiles) << 4);
+        // (the largest cluster at every context length: with fewer CTAs the kernel itself is faster on a short
+        // context - no merge - but the GEMM behind, launched early onto the SMs this grid leaves free, crowds there:
+        // measured, the iteration takes as long)
+        if (c_max >= 1) return 2 | (c_max << 4);
     }
     const int n_mtiles = (rows + 15) / 16;
     if (n_mtiles > 2) return 0;
@@ -1434,7 +1406,7 @@ static int attention_t5(scd_session *s, AttnParams &p, int C, cudaStream_t st)
     int G = 1;
     const T5Kernel fn = t5_kernel(dh, rows, &G);
     const size_t tile_bytes = (size_t)TK * dh * 2;                // one K or V slot
-    const size_t merge_bytes = (size_t)128 * (dh + 4 + 8) * sizeof(float);
+    const size_t merge_bytes = (size_t)128 * (dh + 4 + 4) * sizeof(float);
     // All the shared memory a CTA can have: no CTA of another kernel fits beside this one, so the tensor
     // memory - all 512 columns - is never contended for (see the kernel's header).
     // Behind the rings: the rotated queries on their way to tensor memory, then the window's K and V tiles.
