@@ -136,7 +136,9 @@ int scd_free_model(scd_model_t *model);
  * sequence length; its loop variables i, t, the drafts X and the draft distributions p^(t)).
  * A session holds the KV cache (paged), the window state (drafts, draft distributions, position
  * and iteration counters - all resident on the device) and scratch activations for one decode
- * batch. Allocates device memory (cudaMalloc); free with scd_session_free. */
+ * batch. Allocates device memory (cudaMalloc); free with scd_session_free. bf16 models: a forward
+ * carries S*B*L window rows; the weight GEMMs take them in blocks of 256 (one pass over the weights
+ * per block), and at most 1024 rows are accepted (SCD_ERR_CAPACITY beyond). */
 int scd_session_create(scd_model_t *model, const scd_decode_config_t *cfg, scd_session_t **out);
 int scd_session_free(scd_session_t *session);
 

@@ -255,8 +255,8 @@ int scd_session_create(scd_model_t *m, const scd_decode_config_t *cfg, scd_sessi
     // rows one forward may carry per stream-sequence: the window, or a prefill chunk
     s->chunk = std::max(s->L, std::max(1, std::min(128, 256 / s->Q)));
     s->rows_cap = s->Q * s->chunk;
-    if (c.dtype == SCD_BF16 && s->rows_cap > 256) {
-        set_last_error("bf16 sessions carry at most 256 rows per forward (S*B*L = %d)", s->Q * s->L);
+    if (c.dtype == SCD_BF16 && s->rows_cap > 1024) {
+        set_last_error("bf16 sessions carry at most 1024 rows per forward (S*B*L = %d)", s->Q * s->L);
         delete s;
         return SCD_ERR_CAPACITY;
     }

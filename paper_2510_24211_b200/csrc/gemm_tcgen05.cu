@@ -676,12 +676,13 @@ int make_map(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t K, uint3
 }
 
 // Two-plane activation buffer [2][rows][K] bf16: box = 64 (K) x box_rows x both planes, 128-byte swizzle.
-int make_map_planes(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t K, uint32_t box_rows)
+// (rows: rows of a plane that the map covers from ptr on; plane_rows: rows from one plane to the other)
+int make_map_planes(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t plane_rows, uint64_t K, uint32_t box_rows)
 {
     EncodeTiledFn fn = encode_fn();
     SCD_REQUIRE(fn, SCD_ERR_CUDA, "cuTensorMapEncodeTiled entry point not found");
     cuuint64_t dims[3] = {K, rows, 2};
-    cuuint64_t strides[2] = {K * 2, rows * K * 2};
+    cuuint64_t strides[2] = {K * 2, plane_rows * K * 2};
     cuuint32_t box[3] = {BLOCK_K, box_rows, 2};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr,
@@ -791,16 +792,17 @@ struct SessionGemm {                 // activation-side tensor maps of a session
     std::map<std::tuple<const void *, int, int>, CUtensorMap> xmaps;
 };
 
-// (planes = 2: both planes of an activation buffer in one map; 1: its hi plane alone)
-int x_map(scd_session *s, const void *buf, int K, int nbox, int planes, CUtensorMap *out)
+// (planes = 2: both planes of an activation buffer in one map; 1: its hi plane alone; m0: first row the map covers)
+int x_map(scd_session *s, const void *buf, int K, int nbox, int planes, int m0, CUtensorMap *out)
 {
     SessionGemm *sg = (SessionGemm *)s->gemm_state;
+    buf = (const __nv_bfloat16 *)buf + (size_t)m0 * K;
     auto key = std::make_tuple(buf, K, nbox * 4 + planes);
     auto it = sg->xmaps.find(key);
     if (it == sg->xmaps.end()) {
         CUtensorMap m;
-        int rc = planes == 2 ? make_map_planes(&m, buf, (uint64_t)s->rows_cap, (uint64_t)K, (uint32_t)nbox)
-                             : make_map(&m, buf, (uint64_t)s->rows_cap, (uint64_t)K, (uint32_t)nbox);
+        int rc = planes == 2 ? make_map_planes(&m, buf, (uint64_t)(s->rows_cap - m0), (uint64_t)s->rows_cap, (uint64_t)K, (uint32_t)nbox)
+                             : make_map(&m, buf, (uint64_t)(s->rows_cap - m0), (uint64_t)K, (uint32_t)nbox);
         if (rc != SCD_OK) return rc;
         it = sg->xmaps.emplace(key, m).first;
     }
@@ -830,8 +832,9 @@ int w_map(GemmPlan *plan, const Segment &sg, int box_rows, CUtensorMap *out)
 
 // x_planes: 2 = multiply with both planes of x, 1 = with its hi plane alone (where the output is rounded to
 // bf16 right away - Q, K, V - or is the last stage - the logits - the remainder plane buys nothing)
-int run_gemm(scd_session *s, int kind, const Segment *segs, int n_seg, int epi, const void *x, int K, int rows,
-             void *out, int ldo, const NormIn *nin, const NormOut *nout, int x_planes, cudaStream_t st)
+// (the window rows m0 .. m0 + rows - 1, at most 256: one accumulator holds all rows of a weight tile)
+int run_gemm_rows(scd_session *s, int kind, const Segment *segs, int n_seg, int epi, const void *x, int K, int m0, int rows,
+                  void *out, int ldo, const NormIn *nin, const NormOut *nout, int x_planes, cudaStream_t st)
 {
     GemmPlan *plan = (GemmPlan *)s->model->gemm_plan;
     const bool pair = epi == EPI_SWIGLU;
@@ -859,24 +862,39 @@ int run_gemm(scd_session *s, int kind, const Segment *segs, int n_seg, int epi, 
     p.stages = choose_stages(p.nbox, p.x_planes, (p.k_blocks + p.k_splits - 1) / p.k_splits,
                              tiles * p.k_splits <= 2 * plan->sm_count, plan->forced_stages);
     p.epi = epi;
-    p.out = out;
+    // everything indexed by window row starts at row m0
+    const size_t out_elem = (epi == EPI_BF16 || epi == EPI_SWIGLU) ? 2 : 4;
+    p.out = (char *)out + (size_t)m0 * ldo * out_elem;
     p.ldo = ldo;
     p.ss_stride = s->rows_cap;
     if (nin && nin->ss) {
-        p.ss_in = nin->ss; p.ss_parts = nin->parts;
+        p.ss_in = nin->ss + m0; p.ss_parts = nin->parts;
         p.inv_k = 1.0f / (float)K; p.eps = s->model->cfg.rms_eps;
     }
     if (nout && nout->xg) {
         SCD_REQUIRE(tiles <= s->ss_parts_cap, SCD_ERR_SHAPE, "norm statistics: %d tiles > %d", tiles, s->ss_parts_cap);
-        p.gain_next = (const __nv_bfloat16 *)nout->gain; p.xg_out = (__nv_bfloat16 *)nout->xg; p.ss_out = nout->ss;
+        p.gain_next = (const __nv_bfloat16 *)nout->gain;
+        p.xg_out = (__nv_bfloat16 *)nout->xg + (size_t)m0 * ldo;
+        p.ss_out = nout->ss + m0;
     }
-    int rc = x_map(s, x, K, p.nbox, p.x_planes, &p.tmap_x);
+    int rc = x_map(s, x, K, p.nbox, p.x_planes, m0, &p.tmap_x);
     if (rc != SCD_OK) return rc;
     p.err = (int *)s->gemm_ws;
     p.skip = s->skip_now;
     p.stamp = take_stamp_slot();
     g_last_tiles = tiles;
     return launch(p, tiles, st);
+}
+
+// More than 256 window rows: one pass over the weights per block of 256 rows.
+int run_gemm(scd_session *s, int kind, const Segment *segs, int n_seg, int epi, const void *x, int K, int rows,
+             void *out, int ldo, const NormIn *nin, const NormOut *nout, int x_planes, cudaStream_t st)
+{
+    for (int m0 = 0; m0 < rows; m0 += 256) {
+        const int rc = run_gemm_rows(s, kind, segs, n_seg, epi, x, K, m0, std::min(256, rows - m0), out, ldo, nin, nout, x_planes, st);
+        if (rc != SCD_OK) return rc;
+    }
+    return SCD_OK;
 }
 
 }  // namespace

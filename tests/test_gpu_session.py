@@ -224,9 +224,19 @@ def test_step_replay_wide_window_ragged_batch_bf16():
     _replay_case(MID_BF16_D64, oracle.MODE_SCD_MC, B=3, L=48, P=66, n_new=120, top_k=60, seed=17, page=64)
 
 
-def test_step_replay_four_cfg_pairs_fill_the_row_limit():
-    # B = 4 with guidance at L = 32: 256 window rows in one forward, the most a bf16 session carries
+def test_step_replay_four_cfg_pairs_fill_one_row_block():
+    # B = 4 with guidance at L = 32: 256 window rows, the most one GEMM launch carries
     _replay_case(MID_BF16_D64, oracle.MODE_SCD_MC, B=4, L=32, P=40, n_new=70, top_k=40, lam=1.5, seed=23, page=64)
+
+
+def test_step_replay_more_rows_than_one_gemm_block():
+    # B = 5 with guidance at L = 32: 320 window rows, two passes over the weights per GEMM (256 + 64 rows);
+    # and a session beyond the 1024 rows that are accepted
+    _replay_case(MID_BF16_D64, oracle.MODE_SCD_MC, B=5, L=32, P=40, n_new=50, top_k=40, lam=1.5, seed=29, page=64)
+    gm, _ = _models(MID_BF16_D64, max_seq=128, seed=11, std=0.3, page=64)
+    with pytest.raises(scd.ScdError) as e:
+        scd.Session(gm, scd.decode_config(batch=17, window_L=32, cfg_lambda=1.5, allowed_hi=MID_BF16_D64["vocab_out"]))
+    assert e.value.code == scd.SCD_ERR_CAPACITY
 
 
 def test_autotune_keeps_state_and_parity():
