@@ -125,6 +125,12 @@ def test_step_replay_bf16_tensor_core_attention_cfg_batch(att_min_ctx):
                  page=64, att_min_ctx=att_min_ctx)
 
 
+def test_step_replay_attention_kernel_changes_inside_a_generation():
+    # the committed context passes 512 positions while the sequence is generated: the captured iteration is built
+    # again with the tcgen05 attention kernel in place of the mma.sync one, and the decisions still replay
+    _replay_case(MID_BF16_D64, oracle.MODE_SCD_MC, B=1, L=16, P=490, n_new=80, top_k=40, seed=31, page=64)
+
+
 def _replay_case(shape, mode, B, L, P, n_new, top_k, lam=0.0, temperature=1.0, seed=0, lo=0, hi=None,
                  row_period=0, eol_id=0, std=0.3, page=16, alpha=1.0, top_p=0.0, autotune=False, gm=None,
                  att_min_ctx=None):
