@@ -24,12 +24,12 @@ enum { SCD_PROF_EMBED = 0, SCD_PROF_RMSNORM, SCD_PROF_GEMM_QKV, SCD_PROF_ROPE_KV
 int scd_step_profile(scd_session_t *session, float *ms_by_class, int32_t *launches_by_class,
                      void *stream);
 
-/* scd_session_attention_min_ctx: the decoding steps of a bf16 session use the tcgen05 attention
- * kernel (Sec. 4.3: the window's attention over the committed context) once every live sequence is
- * known to have at least min_ctx committed positions, and the mma.sync kernel below that; the
- * default is 512. min_ctx = 0 selects the tcgen05 kernel for every step, a negative value never.
- * Both kernels compute the same attention; their fp32 additions differ in order. Takes effect at the
- * next scd_step. Errors: SCD_ERR_ARG for a null session. */
+/* scd_session_attention_min_ctx: the forwards of a bf16 session (decoding steps, prefill chunks, explicit
+ * windows) use the tcgen05 attention kernel (Sec. 4.3: the window's attention over the committed
+ * context) once every live sequence is known to hold at least min_ctx committed positions, and the
+ * mma.sync kernel below that; the default is 512. min_ctx = 0 selects the tcgen05 kernel for every
+ * forward, a negative value never. Both kernels compute the same attention; their fp32 additions
+ * differ in order. Takes effect at the next forward. Errors: SCD_ERR_ARG for a null session. */
 int scd_session_attention_min_ctx(scd_session_t *session, int64_t min_ctx);
 
 /* scd_kernel_launches: number of CUDA kernels this process has enqueued through the library. */

@@ -108,7 +108,7 @@ void drop_step_graph(scd_session *s)
 int launch_step(scd_session *s, cudaStream_t st)
 {
     // the captured launches carry the attention variant: capture again when it changes (once per generation)
-    const int variant = s->attn_plan ? attention_tc_variant(s, s->L) : 0;
+    const int variant = s->attn_plan ? attention_tc_variant(s, s->L, s->ctx_floor) : 0;
     if (variant != s->att_variant) { s->att_variant = variant; drop_step_graph(s); }
     struct Advance { scd_session *s; ~Advance() { s->ctx_floor += 1; } } advance{s};   // every iteration commits >= 1 token
     if (s->step_graph_off) return enqueue_step(s, st);

@@ -1374,18 +1374,19 @@ static int t5_max_cluster(const scd_session *s, AttnPlan *plan, int rows)
     return best;
 }
 
-// Low 4 bits: 0 = one warp per query tile; 1 = two warps per query tile; 2 = the tcgen05 kernel (decoding steps only:
-// at most 128 query rows per KV head, the units fit one wave), with its cluster size in the bits above. The choice
-// follows the host's floor of the context length; a captured iteration is built for one value of it.
-int attention_tc_variant(const scd_session *s, int Mq)
+// Low 4 bits: 0 = one warp per query tile; 1 = two warps per query tile; 2 = the tcgen05 kernel (at most 128 query
+// rows per KV head, the units fit one wave), with its cluster size in the bits above. The choice
+// follows `ctx`, the committed positions every live sequence is known to hold: the host's floor of it for a decoding
+// step (a captured iteration is built for one value of the choice), the chunk's first position for a prefill chunk.
+int attention_tc_variant(const scd_session *s, int Mq, long long ctx)
 {
     const scd_model_config_t &c = s->model->cfg;
     AttnPlan *plan = (AttnPlan *)s->attn_plan;
     if (!plan) return 0;
     const int rows = Mq * (c.n_heads / c.n_kv_heads);
-    const long long tiles = (std::max(0ll, s->ctx_floor) + TK - 1) / TK;
+    const long long tiles = (std::max(0ll, ctx) + TK - 1) / TK;
     if (rows <= 128 && s->Q * c.n_kv_heads <= plan->sm_count && (c.max_seq + TK - 1) / TK <= T5_MAX_TILES && s->att_t5_min_ctx >= 0 &&
-        s->ctx_floor >= s->att_t5_min_ctx) {
+        ctx >= s->att_t5_min_ctx) {
         const int c_max = t5_max_cluster(s, plan, rows);
         // (the largest cluster at every context length: with fewer CTAs the kernel itself is faster on a short
         // context - no merge - but the GEMM behind, launched early onto the SMs this grid leaves free, crowds there:
@@ -1462,7 +1463,7 @@ int attention_tc(scd_session *s, int layer, int Mq, int pos_override, cudaStream
     p.max_seq = c.max_seq; p.pos_override = pos_override;
     p.n_mtiles = (Mq * p.n_rep + 15) / 16;
     p.qscale = 1.4426950408889634f / sqrtf((float)c.head_dim);
-    const int variant = pos_override < 0 ? attention_tc_variant(s, Mq) : 0;
+    const int variant = attention_tc_variant(s, Mq, pos_override >= 0 ? (long long)pos_override : s->ctx_floor);
     if ((variant & 15) == 2) return attention_t5(s, p, variant >> 4, st);
     const int units = s->Q * c.n_kv_heads;
     // split-KV over a cluster: up to two CTAs per SM over the whole grid, a power of two (measured:

@@ -41,7 +41,7 @@ void attention_session_release(scd_session *s);
 int attention_tc(scd_session *s, int layer, int Mq, int pos_override, cudaStream_t st);
 // whether the next window forward of the session (Mq rows per stream-sequence) takes the kernel
 // variant for long contexts; a captured iteration is valid only while this does not change
-int attention_tc_variant(const scd_session *s, int Mq);
+int attention_tc_variant(const scd_session *s, int Mq, long long ctx);
 
 // per-session state (activation tensor maps, device error word); bf16 sessions only
 int gemm_session_prepare(scd_session *s);
