@@ -84,7 +84,8 @@ def test_step_replay_long_vocabulary_rows(mode, V, top_k, top_p):
 
 
 # ---- KV cache after partial accepts --------------------------------------------------------------------
-def test_bf16_logits_after_partial_accepts_match_oracle_forward():
+@pytest.mark.parametrize("att_min_ctx", [-1, 0])        # the mma.sync attention kernel, the tcgen05 one
+def test_bf16_logits_after_partial_accepts_match_oracle_forward(att_min_ctx):
     """A stale or misplaced K/V row left behind by an accept or a reject would change the logits of
     every later iteration. Here the GPU session runs on its own (CUDA-graph iterations, CFG pair,
     two sequences, pages of 64 tokens crossed during generation); afterwards the oracle's forward is
@@ -105,6 +106,7 @@ def test_bf16_logits_after_partial_accepts_match_oracle_forward():
     cfg = scd.decode_config(mode=scd.SCD_MODE_SCD_MC, batch=B, window_L=L, top_k=4, cfg_lambda=1.5, seed=3,
                             allowed_hi=shape["vocab_out"])
     sess = scd.Session(gm, cfg)
+    sess.scd_session_attention_min_ctx(att_min_ctx)
     sess.scd_prefill(np.concatenate([cond, uncond]), n_new=n_new)
     rec = []
     n_total = P + n_new
