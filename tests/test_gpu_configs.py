@@ -44,8 +44,8 @@ def test_workload_layer_shape_forward_matches_oracle(name):
 
 
 # ---- full depth -------------------------------------------------------------------------------------
-@pytest.mark.parametrize("name,rows", [("llamagen_xl", 32), ("lumina_7b", 32)])
-def test_full_depth_window_logits_match_oracle(name, rows):
+@pytest.mark.parametrize("name,rows,att_min_ctx", [("llamagen_xl", 32, -1), ("lumina_7b", 32, -1), ("lumina_7b", 32, 0)])
+def test_full_depth_window_logits_match_oracle(name, rows, att_min_ctx):
     """All layers of the workload's decoder, one window on top of a short prompt: the error of the bf16
     path (activations rounded to bf16 between kernels, fp32 accumulation) has the whole depth to grow."""
     shape = synth.WORKLOADS[name]
@@ -57,13 +57,14 @@ def test_full_depth_window_logits_match_oracle(name, rows):
     rng = np.random.default_rng(31)
     prompt = rng.integers(0, shape["vocab_in"], size=(1, P)).astype(np.int32)
     sess = scd.Session(gm, scd.decode_config(batch=1, window_L=rows, allowed_hi=shape["vocab_out"]))
+    sess.scd_session_attention_min_ctx(att_min_ctx)        # -1: the mma.sync attention kernel, 0: the tcgen05 one
     sess.scd_prefill(prompt, n_new=rows + 4)
     om.forward(prompt[0, :-1], 0)
     ids = np.concatenate([prompt[0, -1:], rng.integers(0, shape["vocab_in"], size=rows - 1)]).astype(np.int32)
     logits, hidden = sess.scd_forward_window(torch.from_numpy(ids[None]).cuda(), want_hidden=True)
     ref_logits, ref_hidden = om.forward(ids, P - 1, want_hidden=True)
     e_h, e_l = _rel(hidden[0].cpu().numpy(), ref_hidden), _rel(logits[0].cpu().numpy(), ref_logits)
-    print(f"\n{name}: {shape['n_layers']} layers, max-relative error hidden {e_h:.3e}, logits {e_l:.3e}")
+    print(f"\n{name}: {shape['n_layers']} layers, attention min_ctx {att_min_ctx}, max-relative error hidden {e_h:.3e}, logits {e_l:.3e}")
     assert e_h <= 3e-2 and e_l <= 3e-2
 
 
